@@ -1,0 +1,213 @@
+// CPU oracle for the MoE FFN layer forward with a hot/cold expert split.
+//
+// TEST INFRASTRUCTURE ONLY.  This is the plain, slow, scalar fp64 statement of
+// what the layer computes.  It exists to check the CUDA library and to be timed
+// as a CPU baseline; nothing in the product path may call it.  It shares no
+// code with the CUDA sources.
+//
+// What it follows (MoNDE, Section 2.1 "Mixture of Experts", Fig. 1): a gating
+// network gives, per token, a probability distribution over the E experts (the
+// token x expert score map); each token is routed to its top-k experts; each
+// expert is two linear layers with one activation between (ReLU or GeLU,
+// Section 3.4 "Host Interface"); expert outputs are combined and put back in
+// the original token order.  Routing is drop-less and padding-less (Section 4.1
+// "Implementation").  Experts are labelled hot or cold by how many tokens they
+// receive (Section 2.2 "Expert Skew and Load Imbalance"); experts with no token
+// are not activated (Section 3.3, Eq. 5).  The labelling never changes the
+// arithmetic: hot and cold experts compute the same FFN.
+//
+// Readings where the paper is silent are listed in the design notes; the ones
+// that matter here: the gate is linear (+ optional bias) followed by a softmax
+// over all E experts; selection compares logits, best first, exact ties to the
+// smaller expert id; combine weights are the softmax probabilities, optionally
+// renormalised over the k selected; GeLU is the erf form; experts ascending and
+// assignments ascending inside an expert fix the one permutation that is
+// reported; all arithmetic is fp64 on the exact input values.
+//
+// Pins (tests that tie this file to something other than itself): E=1 dense
+// reduction against a library matmul, one-hot gate bias, dense-masked
+// restatement with brute-force subset choice, identity-weights closed form,
+// library sort for top-k, uniform-logit tie case, softmax-over-selected
+// identity, bincount / cumsum / stable argsort, a hand-worked example and
+// tabulated Phi(v) values for GeLU.  Absolute output values have no worked
+// example in the paper; they are pinned only through those reductions.
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <thread>
+#include <vector>
+
+#include <sched.h>
+
+namespace {
+
+enum { DT_F32 = 0, DT_BF16 = 1 };
+enum { ACT_RELU = 0, ACT_GELU = 1 };
+
+inline double widen(const void* base, int64_t i, int dtype) {
+    if (dtype == DT_F32) return static_cast<double>(static_cast<const float*>(base)[i]);
+    uint32_t bits = static_cast<uint32_t>(static_cast<const uint16_t*>(base)[i]) << 16;
+    float v;
+    std::memcpy(&v, &bits, sizeof v);
+    return static_cast<double>(v);
+}
+
+inline double activation(double v, int act) {
+    if (act == ACT_RELU) return v > 0.0 ? v : 0.0;
+    return 0.5 * v * (1.0 + std::erf(v / std::sqrt(2.0)));
+}
+
+int usable_cores() {
+    cpu_set_t set;
+    CPU_ZERO(&set);
+    if (sched_getaffinity(0, sizeof set, &set) == 0) {
+        int n = CPU_COUNT(&set);
+        if (n > 0) return n;
+    }
+    unsigned h = std::thread::hardware_concurrency();
+    return h ? static_cast<int>(h) : 1;
+}
+
+template <class F>
+void for_rows(int64_t n, int nthreads, F body) {
+    if (nthreads <= 0) nthreads = usable_cores();
+    if (nthreads > n) nthreads = static_cast<int>(n > 0 ? n : 1);
+    if (nthreads <= 1) {
+        for (int64_t r = 0; r < n; ++r) body(r);
+        return;
+    }
+    std::vector<std::thread> pool;
+    for (int w = 0; w < nthreads; ++w)
+        pool.emplace_back([=]() { for (int64_t r = w; r < n; r += nthreads) body(r); });
+    for (auto& t : pool) t.join();
+}
+
+}  // namespace
+
+extern "C" {
+
+int oracle_usable_cores() { return usable_cores(); }
+
+// Gate, softmax, top-k, histogram, classification, scan (Section 2.1; Section 2.2
+// for hot/cold; Eq. 5 for "activated").
+//   x [T,d], Wg [E,d] in `dtype`; bg [E] fp32 or null.
+//   logits, probs [T,E] fp64 (nullable); topk_idx [T,k] int32; topk_w [T,k] fp64;
+//   counts [E]; offsets [E+1]; cls [E] (0 inactive, 1 cold, 2 hot);
+//   hot_ids, cold_ids [E] (first n entries valid, ascending); n_hot_cold [2].
+void oracle_route(int T, int d, int E, int k, int renormalize, int hot_threshold, int dtype,
+                  const void* x, const void* Wg, const float* bg,
+                  double* logits, double* probs, int32_t* topk_idx, double* topk_w,
+                  int32_t* counts, int32_t* offsets, uint8_t* cls,
+                  int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold) {
+    std::vector<double> l(E), p(E);
+    std::vector<char> taken(E);
+    for (int e = 0; e < E; ++e) counts[e] = 0;
+    for (int t = 0; t < T; ++t) {
+        for (int e = 0; e < E; ++e) {
+            double acc = bg ? static_cast<double>(bg[e]) : 0.0;
+            for (int i = 0; i < d; ++i)
+                acc += widen(x, static_cast<int64_t>(t) * d + i, dtype) *
+                       widen(Wg, static_cast<int64_t>(e) * d + i, dtype);
+            l[e] = acc;
+        }
+        double lmax = l[0];
+        for (int e = 1; e < E; ++e) lmax = std::max(lmax, l[e]);
+        double denom = 0.0;
+        for (int e = 0; e < E; ++e) { p[e] = std::exp(l[e] - lmax); denom += p[e]; }
+        for (int e = 0; e < E; ++e) p[e] /= denom;
+
+        std::fill(taken.begin(), taken.end(), 0);
+        double selected_mass = 0.0;
+        for (int j = 0; j < k; ++j) {
+            int best = -1;
+            for (int e = 0; e < E; ++e)
+                if (!taken[e] && (best < 0 || l[e] > l[best])) best = e;
+            taken[best] = 1;
+            topk_idx[static_cast<int64_t>(t) * k + j] = best;
+            selected_mass += p[best];
+            counts[best] += 1;
+        }
+        for (int j = 0; j < k; ++j) {
+            double pj = p[topk_idx[static_cast<int64_t>(t) * k + j]];
+            topk_w[static_cast<int64_t>(t) * k + j] = renormalize ? pj / selected_mass : pj;
+        }
+        if (logits) for (int e = 0; e < E; ++e) logits[static_cast<int64_t>(t) * E + e] = l[e];
+        if (probs)  for (int e = 0; e < E; ++e) probs[static_cast<int64_t>(t) * E + e] = p[e];
+    }
+    int n_hot = 0, n_cold = 0;
+    offsets[0] = 0;
+    for (int e = 0; e < E; ++e) {
+        offsets[e + 1] = offsets[e] + counts[e];
+        if (counts[e] == 0) cls[e] = 0;
+        else if (counts[e] >= hot_threshold) { cls[e] = 2; hot_ids[n_hot++] = e; }
+        else { cls[e] = 1; cold_ids[n_cold++] = e; }
+    }
+    n_hot_cold[0] = n_hot;
+    n_hot_cold[1] = n_cold;
+}
+
+// Expert-contiguous order: experts ascending, and inside an expert the flat
+// assignment ids a = t*k + j ascending.  perm[pos] = a, inv_perm[a] = pos,
+// x_perm[pos,:] = x[a / k,:] (byte copy).  Drop-less, padding-less (Section 4.1).
+void oracle_permute(int T, int d, int E, int k, int elem_bytes,
+                    const void* x, const int32_t* topk_idx, const int32_t* offsets,
+                    int32_t* perm, int32_t* inv_perm, void* x_perm) {
+    std::vector<int32_t> seen(E, 0);
+    const int64_t A = static_cast<int64_t>(T) * k;
+    const size_t row = static_cast<size_t>(d) * elem_bytes;
+    for (int64_t a = 0; a < A; ++a) {
+        int e = topk_idx[a];
+        int32_t pos = offsets[e] + seen[e];
+        seen[e] += 1;
+        perm[pos] = static_cast<int32_t>(a);
+        inv_perm[a] = pos;
+        if (x_perm)
+            std::memcpy(static_cast<char*>(x_perm) + static_cast<size_t>(pos) * row,
+                        static_cast<const char*>(x) + static_cast<size_t>(a / k) * row, row);
+    }
+}
+
+// Expert FFN for a list of rows (Section 2.1: two linear layers, one activation).
+//   rows [n,d] in `dtype`; row_expert [n]; W1 [*,f,d], b1 [*,f], W2 [*,d,f], b2 [*,d]
+//   in `dtype` (biases nullable); h_out [n,f] fp64 (nullable); y_out [n,d] fp64.
+void oracle_expert_ffn(int64_t n, int d, int f, int act, int dtype,
+                       const void* rows, const int32_t* row_expert,
+                       const void* W1, const void* b1, const void* W2, const void* b2,
+                       double* h_out, double* y_out, int nthreads) {
+    for_rows(n, nthreads, [=](int64_t r) {
+        const int64_t e = row_expert[r];
+        std::vector<double> xr(d), h(f);
+        for (int i = 0; i < d; ++i) xr[i] = widen(rows, r * d + i, dtype);
+        for (int m = 0; m < f; ++m) {
+            double acc = b1 ? widen(b1, e * f + m, dtype) : 0.0;
+            const int64_t w = (e * f + m) * static_cast<int64_t>(d);
+            for (int i = 0; i < d; ++i) acc += xr[i] * widen(W1, w + i, dtype);
+            h[m] = activation(acc, act);
+        }
+        if (h_out) for (int m = 0; m < f; ++m) h_out[r * f + m] = h[m];
+        for (int c = 0; c < d; ++c) {
+            double acc = b2 ? widen(b2, e * d + c, dtype) : 0.0;
+            const int64_t w = (e * d + c) * static_cast<int64_t>(f);
+            for (int m = 0; m < f; ++m) acc += h[m] * widen(W2, w + m, dtype);
+            y_out[r * d + c] = acc;
+        }
+    });
+}
+
+// Gate-weighted combine back to token order (Section 2.1), slots ascending.
+void oracle_combine(int T, int d, int k, const double* y_perm, const int32_t* inv_perm,
+                    const double* topk_w, double* out) {
+    for (int t = 0; t < T; ++t)
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int j = 0; j < k; ++j) {
+                const int64_t a = static_cast<int64_t>(t) * k + j;
+                acc += topk_w[a] * y_perm[static_cast<int64_t>(inv_perm[a]) * d + c];
+            }
+            out[static_cast<int64_t>(t) * d + c] = acc;
+        }
+}
+
+}  // extern "C"
