@@ -1,0 +1,338 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE FFN layer forward (route -> permute -> hot/cold expert FFN ->
+combine) on synthetic Switch / NLLB-shaped workloads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1|C2|C3] [--impl ours|reference]
+
+One JSON line on stdout (rank 0).  A step is one pass of the whole layer over one
+batch of T tokens.  `value` is tokens/s with inputs resident in HBM; `e2e` is the
+same layer called with the step's tokens in pinned host memory (H2D copy of x and
+D2H copy of the output inside the timed region).  `roofline` describes the dominant
+call (the expert FFN) from CUDA events taken inside the timed region; `cpu_baseline`
+is the fp64 CPU oracle timed on this host on a bounded sample of the same workload.
+
+With N > 1 (launched under torchrun, one rank per GPU) every rank runs an independent
+replica of the layer on its own batch: the path has no exchange step on one node, so
+no collective is on the data path; only the barrier and the max-over-ranks of the
+device time use torch.distributed.
+
+`--impl reference` times the CPU oracle (the only reference implementation there is
+for this paper: it published no code) on the host cores, on a bounded sample per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2405_18832_b200 import synthetic as S  # noqa: E402
+
+METRIC = "moe_ffn_layer_tokens_per_s"
+UNIT = "tokens/s"
+
+# DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures
+# summarised under profiles/ (None until a capture exists for that workload).
+NCU_TRAFFIC_BYTES = {"C1": None, "C2": None, "C3": None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        m = json.load(open(path))
+        return dict(hbm_gbs=float(m["hbm_gbs"]), bf16_tflops=float(m["bf16_tflops"]),
+                    bf16_tflops_sustained=float(m.get("bf16_tflops_sustained", m["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def ffn_algorithmic_bytes(p: S.Problem, counts: np.ndarray) -> float:
+    """Bytes the expert FFN must move: each activated expert's W1 and W2 once (Eq. 1 of the
+    paper per expert: 2*d_model*d_ff parameters), x_perm read, h written and read, y_perm
+    written, for every routed row."""
+    s = p.elem_bytes
+    active = int((counts > 0).sum())
+    A = int(counts.sum())
+    return active * 2.0 * p.d_model * p.d_ff * s + A * (2.0 * p.d_model + 2.0 * p.d_ff) * s
+
+
+def ffn_flops(p: S.Problem, counts: np.ndarray) -> float:
+    return 4.0 * float(counts.sum()) * p.d_model * p.d_ff
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", gpu_id, "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [c.strip() for c in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample_run(w: S.Workload, host, n_tokens: int, nthreads: int = 0):
+    """Whole layer through the CPU oracle on the first n_tokens tokens; returns seconds."""
+    import oracle
+    p = w.problem
+    t0 = time.perf_counter()
+    oracle.moe_layer(host["x"][:n_tokens], host["Wg"], host["bg"], host["W1"], host["b1"], host["W2"], host["b2"],
+                     p.top_k, p.renormalize, p.hot_threshold, p.act, nthreads)
+    return time.perf_counter() - t0
+
+
+def host_inputs(g):
+    return {k: S.as_numpy(v) for k, v in g.items()}
+
+
+def pick_sample_tokens(w, host, target_s: float) -> int:
+    import oracle
+    cores = oracle.usable_cores()
+    probe = min(w.problem.T, max(cores, 8))
+    dt = oracle_sample_run(w, host, probe)
+    n = int(probe * target_s / max(dt, 1e-6))
+    return max(1, min(w.problem.T, n))
+
+
+def generate_inputs(w: S.Workload, device):
+    g = S.generate(w, with_weights=False)
+    gw = S.generate(w, weights_device=device)
+    for k in ("W1", "W2", "b1", "b2"):
+        g[k] = gw[k]
+    return g
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    host = host_inputs(generate_inputs(w, dev))
+    cores = oracle.usable_cores()
+    per_step = max(0.5, min(5.0, 150.0 / max(1, args.steps + args.warmup)))
+    n_tok = pick_sample_tokens(w, host, per_step)
+    for _ in range(args.warmup):
+        oracle_sample_run(w, host, n_tok)
+    t = [oracle_sample_run(w, host, n_tok) for _ in range(args.steps)]
+    sec = sum(t) / len(t)
+    value = n_tok / sec
+    sample = f"whole layer on the first {n_tok} of {w.problem.T} tokens per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def workload_config(w):
+    p = w.problem
+    return {"workload": f"{w.name}: E={p.E} top-{p.top_k} d_model={p.d_model} d_ff={p.d_ff} T={p.T} {p.dtype} "
+                        f"{p.act} hot_threshold={p.hot_threshold} zipf_alpha={w.zipf_alpha}",
+            "tokens_per_step_per_gpu": p.T, "seed": w.seed,
+            "l2": "256 MiB scratch write between timed steps (L2 flush); active weights also exceed L2",
+            "parallelism": "independent replicas, one per GPU, no data-path collective"}
+
+
+def run_ours(args, w):
+    from paper_2405_18832_b200 import binding as B
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    p = w.problem
+    if world > 1:   # every replica gets its own batch
+        import dataclasses
+        w = dataclasses.replace(w, seed=w.seed + 1000 * rank)
+    g = generate_inputs(w, dev)
+    d = {k: (None if v is None else v.to(dev)) for k, v in g.items()}
+    buf = B.LayerBuffers(p, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    L = B.lib()
+    has_counter = hasattr(L, "monde_kernel_launches")
+
+    def layer(ev=None):
+        if ev is not None:
+            ev[0].record(stream)
+        B.monde_route(p, d["x"], d["Wg"], d["bg"], buf.topk_idx, buf.topk_w, buf.counts, buf.offsets, buf.cls,
+                      buf.hot_ids, buf.cold_ids, buf.n_hot_cold, None, buf.ws)
+        if ev is not None:
+            ev[1].record(stream)
+        B.monde_permute(p, d["x"], buf.topk_idx, buf.offsets, buf.perm, buf.inv_perm, buf.x_perm, buf.ws)
+        if ev is not None:
+            ev[2].record(stream)
+        B.monde_moe_ffn_fwd(p, buf.x_perm, d["W1"], d["b1"], d["W2"], d["b2"], buf.counts, buf.offsets, buf.cls,
+                            buf.hot_ids, buf.cold_ids, buf.n_hot_cold, buf.y_perm, buf.ws)
+        if ev is not None:
+            ev[3].record(stream)
+        B.monde_combine(p, buf.y_perm, buf.inv_perm, buf.topk_w, buf.out)
+        if ev is not None:
+            ev[4].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        flush.fill_(1)
+        layer()
+    B.monde_poll_device_status(buf.ws)
+    counts = buf.counts.cpu().numpy()
+
+    # ---- timed region: device-resident inputs --------------------------------------
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
+    launches0 = L.monde_kernel_launches() if has_counter else 0
+    wall0 = time.perf_counter()
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)
+        layer(events[i])
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    launches = (L.monde_kernel_launches() - launches0) if has_counter else None
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop()
+    B.monde_poll_device_status(buf.ws)
+    step_ms = [e[0].elapsed_time(e[4]) for e in events]
+    call_ms = [[e[i].elapsed_time(e[i + 1]) for e in events] for i in range(4)]
+    total_ms = sum(step_ms)
+    tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    value = world * p.T / (ms_per_step * 1e-3)
+
+    # ---- end to end: tokens in pinned host memory ----------------------------------
+    x_host = g["x"].pin_memory()
+    out_host = torch.empty((p.T, p.d_model), dtype=p.torch_dtype).pin_memory()
+    for _ in range(3):
+        B.moe_ffn_layer_forward_host(p, x_host, out_host, d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"], buf)
+    e2e_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    for a, b in e2e_ev:
+        flush.fill_(3)
+        a.record(stream)
+        B.moe_ffn_layer_forward_host(p, x_host, out_host, d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"], buf)
+        b.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = sum(a.elapsed_time(b) for a, b in e2e_ev)
+    te = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_value = world * p.T / (float(te.item()) / args.steps * 1e-3)
+    assert torch.equal(out_host, buf.out.cpu())
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    ffn_ms = statistics.mean(call_ms[2])
+    bytes_ffn = ffn_algorithmic_bytes(p, counts)
+    achieved = bytes_ffn / (ffn_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "monde_moe_ffn_fwd (hot + cold expert FFN)", "achieved": achieved,
+                "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                "algorithmic_bytes": bytes_ffn, "ms": ffn_ms,
+                "tflops": ffn_flops(p, counts) / (ffn_ms * 1e-3) / 1e12}
+    layer_floor_ms = (bytes_ffn + (2 * p.A + 2 * p.T) * p.d_model * p.elem_bytes + p.T * p.d_model * p.elem_bytes) \
+        / (peaks["hbm_gbs"] * 1e9) * 1e3
+
+    # ---- CPU baseline: the oracle as it stands, on a bounded sample ------------------
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        import oracle
+        host = host_inputs(g)
+        n_tok = pick_sample_tokens(w, host, 12.0)
+        sec = oracle_sample_run(w, host, n_tok)
+        cpu = {"value": n_tok / sec, "unit": UNIT, "cores": oracle.usable_cores(), "kind": "oracle",
+               "sample": f"whole layer on the first {n_tok} of {p.T} tokens, {sec:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": p.dtype, "data": "synthetic", "config": workload_config(w),
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
+                "d2h_bytes_per_step": out_host.numel() * out_host.element_size()},
+        "gpu_launches": launches,
+        "roofline": roofline, "cpu_baseline": cpu,
+        "calls_ms": {"route": statistics.mean(call_ms[0]), "permute": statistics.mean(call_ms[1]),
+                     "ffn": ffn_ms, "combine": statistics.mean(call_ms[3])},
+        "layer_hbm_floor_ms": layer_floor_ms, "layer_roofline_frac": layer_floor_ms / ms_per_step,
+        "routing": {"active": int((counts > 0).sum()), "hot": int((counts >= p.hot_threshold).sum()),
+                    "max_count": int(counts.max()), "assignments": int(counts.sum())},
+        "wall_s_timed_region": wall,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="C1", choices=["C1", "C2", "C3"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = S.config(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,172 @@
+// extern "C" entry points: argument checks, workspace carving, launches.
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace monde {
+
+int check_problem(const monde_problem* p) {
+    if (p == nullptr) return MONDE_ERR_INVALID_ARG;
+    if (p->T < 0 || p->d_model <= 0 || p->d_ff <= 0 || p->E <= 0 || p->top_k <= 0) return MONDE_ERR_INVALID_ARG;
+    if (p->top_k > p->E) return MONDE_ERR_INVALID_ARG;
+    if (p->dtype != MONDE_F32 && p->dtype != MONDE_BF16) return MONDE_ERR_UNSUPPORTED;
+    if (p->act != MONDE_ACT_RELU && p->act != MONDE_ACT_GELU_ERF) return MONDE_ERR_UNSUPPORTED;
+    if (p->E > kMaxExperts || p->top_k > kMaxTopK) return MONDE_ERR_UNSUPPORTED;
+    const int mult = p->dtype == MONDE_BF16 ? 64 : 4;
+    if (p->d_model % mult != 0 || p->d_ff % mult != 0) return MONDE_ERR_UNSUPPORTED;
+    if (static_cast<int64_t>(p->T) * p->top_k > (1ll << 30)) return MONDE_ERR_UNSUPPORTED;
+    return MONDE_OK;
+}
+
+static std::atomic<long long> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_arch() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MONDE_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return MONDE_ERR_CUDA;
+    return major == 10 ? MONDE_OK : MONDE_ERR_ARCH;
+}
+
+int check_ws(const monde_problem& p, const void* ws, size_t ws_bytes) {
+    if (ws == nullptr || !aligned16(ws)) return MONDE_ERR_INVALID_ARG;
+    if (ws_bytes < ws_layout(p).total) return MONDE_ERR_WORKSPACE;
+    return MONDE_OK;
+}
+
+bool force_simt() {
+    static const bool v = [] {
+        const char* e = std::getenv("MONDE_FFN_IMPL");
+        return e != nullptr && std::strcmp(e, "simt") == 0;
+    }();
+    return v;
+}
+
+}  // namespace
+}  // namespace monde
+
+using namespace monde;
+
+extern "C" {
+
+size_t monde_workspace_bytes(const monde_problem* p) {
+    if (check_problem(p) != MONDE_OK) return 0;
+    return ws_layout(*p).total;
+}
+
+const char* monde_status_string(int status) {
+    switch (status) {
+        case MONDE_OK: return "ok";
+        case MONDE_ERR_INVALID_ARG: return "invalid argument";
+        case MONDE_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case MONDE_ERR_WORKSPACE: return "workspace too small";
+        case MONDE_ERR_ARCH: return "device is not compute capability 10.x";
+        case MONDE_ERR_CUDA: return "CUDA call failed";
+        case MONDE_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+int monde_route(const monde_problem* p, const void* x, const void* Wg, const float* bg,
+                int32_t* topk_idx, float* topk_w, int32_t* counts, int32_t* offsets,
+                uint8_t* cls, int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold,
+                float* probs, void* ws, size_t ws_bytes, void* stream) {
+    int st = check_problem(p);
+    if (st != MONDE_OK) return st;
+    if (!Wg || !counts || !offsets || !cls || !hot_ids || !cold_ids || !n_hot_cold) return MONDE_ERR_INVALID_ARG;
+    if (p->T > 0 && (!x || !topk_idx || !topk_w)) return MONDE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(Wg)) return MONDE_ERR_INVALID_ARG;
+    if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
+    if ((st = check_arch()) != MONDE_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (p->T > 0) {
+        st = launch_route(*p, x, Wg, bg, topk_idx, topk_w, probs, s);
+        if (st != MONDE_OK) return st;
+    }
+    return launch_histogram_classify_scan(*p, topk_idx, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold, s);
+}
+
+int monde_permute(const monde_problem* p, const void* x, const int32_t* topk_idx,
+                  const int32_t* offsets, int32_t* perm, int32_t* inv_perm, void* x_perm,
+                  void* ws, size_t ws_bytes, void* stream) {
+    int st = check_problem(p);
+    if (st != MONDE_OK) return st;
+    if (p->T == 0) return MONDE_OK;
+    if (!x || !topk_idx || !offsets || !perm || !inv_perm || !x_perm) return MONDE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(x_perm)) return MONDE_ERR_INVALID_ARG;
+    if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
+    if ((st = check_arch()) != MONDE_OK) return st;
+    return launch_permute(*p, x, topk_idx, offsets, perm, inv_perm, x_perm, static_cast<cudaStream_t>(stream));
+}
+
+int monde_moe_ffn_fwd(const monde_problem* p, const void* x_perm,
+                      const void* W1, const void* b1, const void* W2, const void* b2,
+                      const int32_t* counts, const int32_t* offsets, const uint8_t* cls,
+                      const int32_t* hot_ids, const int32_t* cold_ids, const int32_t* n_hot_cold,
+                      void* y_perm, void* ws, size_t ws_bytes, void* stream) {
+    int st = check_problem(p);
+    if (st != MONDE_OK) return st;
+    if (p->T == 0) return MONDE_OK;
+    if (!x_perm || !W1 || !W2 || !counts || !offsets || !cls || !hot_ids || !cold_ids || !n_hot_cold || !y_perm)
+        return MONDE_ERR_INVALID_ARG;
+    if (!aligned16(x_perm) || !aligned16(W1) || !aligned16(W2) || !aligned16(y_perm) || !aligned16(b1) ||
+        !aligned16(b2))
+        return MONDE_ERR_INVALID_ARG;
+    if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
+    if ((st = check_arch()) != MONDE_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    void* h = static_cast<char*>(ws) + WsLayout::kHidden;
+    if (p->dtype == MONDE_F32 || force_simt()) {
+        // Same kernel for both classes; the class lists still select the experts.
+        const int32_t* lists[2] = {hot_ids, cold_ids};
+        for (int c = 0; c < 2; ++c) {
+            st = launch_linear_simt(p->dtype, p->act, p->E, p->d_model, p->d_ff, x_perm, W1, b1, offsets,
+                                    lists[c], n_hot_cold + c, h, s);
+            if (st != MONDE_OK) return st;
+            st = launch_linear_simt(p->dtype, -1, p->E, p->d_ff, p->d_model, h, W2, b2, offsets, lists[c],
+                                    n_hot_cold + c, y_perm, s);
+            if (st != MONDE_OK) return st;
+        }
+        return MONDE_OK;
+    }
+    return launch_ffn_bf16(*p, x_perm, W1, b1, W2, b2, counts, offsets, hot_ids, cold_ids, n_hot_cold, y_perm, ws, s);
+}
+
+int monde_combine(const monde_problem* p, const void* y_perm, const int32_t* inv_perm,
+                  const float* topk_w, void* out, void* stream) {
+    int st = check_problem(p);
+    if (st != MONDE_OK) return st;
+    if (p->T == 0) return MONDE_OK;
+    if (!y_perm || !inv_perm || !topk_w || !out) return MONDE_ERR_INVALID_ARG;
+    if (!aligned16(y_perm) || !aligned16(out)) return MONDE_ERR_INVALID_ARG;
+    if ((st = check_arch()) != MONDE_OK) return st;
+    return launch_combine(*p, y_perm, inv_perm, topk_w, out, static_cast<cudaStream_t>(stream));
+}
+
+long long monde_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int monde_poll_device_status(void* ws, void* stream, int32_t* site) {
+    if (ws == nullptr) return MONDE_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t word[2] = {0, 0};
+    if (cudaMemcpyAsync(word, static_cast<char*>(ws) + WsLayout::kStatus, sizeof word, cudaMemcpyDeviceToHost, s) !=
+        cudaSuccess)
+        return MONDE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return MONDE_ERR_CUDA;
+    if (site != nullptr) *site = word[1];
+    if (word[0] != 0) {
+        if (cudaMemsetAsync(static_cast<char*>(ws) + WsLayout::kStatus, 0, sizeof word, s) != cudaSuccess)
+            return MONDE_ERR_CUDA;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return MONDE_ERR_CUDA;
+    }
+    return word[0];
+}
+
+}  // extern "C"

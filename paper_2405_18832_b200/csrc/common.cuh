@@ -1,0 +1,123 @@
+// Shared declarations of the CUDA library: problem checks, workspace layout,
+// element load/convert helpers, launch prototypes.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/monde.h"
+
+namespace monde {
+
+constexpr int kMaxExperts = 256;
+constexpr int kMaxTopK = 8;
+
+// Workspace carving.  Offsets in bytes from the workspace base.
+struct WsLayout {
+    static constexpr size_t kStatus = 0;        // int32 status, int32 site
+    static constexpr size_t kCounters = 1024;   // int32 counters used by the FFN kernels
+    static constexpr size_t kCountersBytes = 15 * 1024;
+    static constexpr size_t kTiles = 16 * 1024; // work lists built on the device
+    static constexpr size_t kTilesBytes = 112 * 1024;
+    static constexpr size_t kHidden = 128 * 1024;  // h [A, d_ff] in the problem dtype
+    size_t hidden_bytes;
+    size_t total;
+};
+
+inline size_t elem_bytes(int dtype) { return dtype == MONDE_BF16 ? 2 : 4; }
+
+inline WsLayout ws_layout(const monde_problem& p) {
+    WsLayout l;
+    size_t A = static_cast<size_t>(p.T) * p.top_k;
+    l.hidden_bytes = (A * p.d_ff * elem_bytes(p.dtype) + 1023) / 1024 * 1024;
+    l.total = WsLayout::kHidden + l.hidden_bytes + 1024;
+    return l;
+}
+
+// MONDE_OK when the problem is inside the stated limits.
+int check_problem(const monde_problem* p);
+
+// ---- element helpers --------------------------------------------------------
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_float(float v);
+template <> __device__ __forceinline__ float from_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) {
+    return __float2bfloat16_rn(v);
+}
+
+// 16-byte vector of elements, unpacked to floats.
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+    static constexpr int N = 4;
+    __device__ static __forceinline__ void load(const float* p, float (&o)[4]) {
+        float4 v = *reinterpret_cast<const float4*>(p);
+        o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+    }
+    __device__ static __forceinline__ void store(float* p, const float (&o)[4]) {
+        *reinterpret_cast<float4*>(p) = make_float4(o[0], o[1], o[2], o[3]);
+    }
+};
+template <> struct Vec16<__nv_bfloat16> {
+    static constexpr int N = 8;
+    __device__ static __forceinline__ void load(const __nv_bfloat16* p, float (&o)[8]) {
+        uint4 v = *reinterpret_cast<const uint4*>(p);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            o[2 * i] = __uint_as_float(w[i] << 16);
+            o[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    __device__ static __forceinline__ void store(__nv_bfloat16* p, const float (&o)[8]) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+__device__ __forceinline__ float apply_act(float v, int act) {
+    if (act == MONDE_ACT_RELU) return fmaxf(v, 0.0f);
+    return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f));
+}
+
+// ---- launch prototypes (each returns a monde_status) -------------------------
+int launch_route(const monde_problem& p, const void* x, const void* Wg, const float* bg,
+                 int32_t* topk_idx, float* topk_w, float* probs, cudaStream_t s);
+int launch_histogram_classify_scan(const monde_problem& p, const int32_t* topk_idx, int32_t* counts,
+                                   int32_t* offsets, uint8_t* cls, int32_t* hot_ids, int32_t* cold_ids,
+                                   int32_t* n_hot_cold, cudaStream_t s);
+int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_idx, const int32_t* offsets,
+                   int32_t* perm, int32_t* inv_perm, void* x_perm, cudaStream_t s);
+int launch_combine(const monde_problem& p, const void* y_perm, const int32_t* inv_perm,
+                   const float* topk_w, void* out, cudaStream_t s);
+
+// Out[r, n] = act?(bias[e, n] + sum_k In[r, k] * W[e, n, k]) for the rows of the experts in
+// `ids[0 .. *n_ids)`; plain CUDA-core kernel (fp32 problems; debugging aid for bf16).
+int launch_linear_simt(int dtype, int act_or_neg1, int E, int K, int N, const void* in, const void* W,
+                       const void* bias, const int32_t* offsets, const int32_t* ids, const int32_t* n_ids,
+                       void* out, cudaStream_t s);
+
+// bf16 problems: hot experts on the tcgen05 grouped GEMM, cold experts on the
+// weight-streaming kernel.
+int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, const void* b1,
+                    const void* W2, const void* b2, const int32_t* counts, const int32_t* offsets,
+                    const int32_t* hot_ids, const int32_t* cold_ids, const int32_t* n_hot_cold,
+                    void* y_perm, void* ws, cudaStream_t s);
+
+// Process-wide count of kernels this library has launched (diagnostic).
+void count_launches(int n);
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? MONDE_OK : MONDE_ERR_CUDA; }
+inline int launched(int n = 1) {
+    count_launches(n);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace monde

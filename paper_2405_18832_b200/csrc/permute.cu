@@ -1,0 +1,118 @@
+// Stable counting-sort permutation of assignments into expert-contiguous order, fused
+// with the row gather.  Deterministic: positions follow from counts alone, never from
+// the order in which threads run.
+// Paper: Section 2.1 (routing to experts); Section 4.1 (drop-less, padding-less).
+#include "common.cuh"
+
+namespace monde {
+
+namespace {
+
+constexpr int kChunk = 128;          // assignments per CTA
+constexpr int kWarps = kChunk / 32;
+
+// CTA c owns assignments [c*kChunk, (c+1)*kChunk).  The number of earlier assignments to
+// each expert is recounted from topk_idx (at most A integers, L2-resident), which keeps
+// the kernel single-pass and free of inter-CTA ordering.
+template <typename T>
+__global__ void __launch_bounds__(kChunk) permute_gather_kernel(
+        int A, int E, int k, int d, const T* __restrict__ x, const int32_t* __restrict__ topk_idx,
+        const int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
+        T* __restrict__ x_perm) {
+    __shared__ int before[kMaxExperts];              // assignments to e in earlier chunks
+    __shared__ int warp_cnt[kWarps][kMaxExperts];    // assignments to e per warp of this chunk
+    __shared__ int row_pos[kChunk];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int first = blockIdx.x * kChunk;
+    for (int e = tid; e < kMaxExperts; e += kChunk) {
+        before[e] = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) warp_cnt[w][e] = 0;
+    }
+    __syncthreads();
+    for (int a = tid; a < first; a += kChunk) atomicAdd(&before[topk_idx[a]], 1);
+    const int a = first + tid;
+    const int e = a < A ? topk_idx[a] : -1;
+    const unsigned same = __match_any_sync(0xffffffffu, e);
+    const int rank_in_warp = __popc(same & ((1u << lane) - 1u));
+    if (e >= 0 && rank_in_warp == 0) warp_cnt[warp][e] = __popc(same);
+    __syncthreads();
+    int pos = -1;
+    if (e >= 0) {
+        pos = offsets[e] + before[e] + rank_in_warp;
+        for (int w = 0; w < warp; ++w) pos += warp_cnt[w][e];
+        perm[pos] = a;
+        inv_perm[a] = pos;
+    }
+    row_pos[tid] = pos;
+    __syncthreads();
+    // Row gather: each warp copies whole rows with 16-byte accesses.
+    constexpr int V = Vec16<T>::N;
+    const int vec_per_row = d / V;
+    for (int r = warp; r < kChunk; r += kWarps) {
+        const int p = row_pos[r];
+        if (p < 0) break;
+        const uint4* src = reinterpret_cast<const uint4*>(x + static_cast<int64_t>((first + r) / k) * d);
+        uint4* dst = reinterpret_cast<uint4*>(x_perm + static_cast<int64_t>(p) * d);
+        for (int i = lane; i < vec_per_row; i += 32) dst[i] = src[i];
+    }
+}
+
+// out[t,:] = sum_j w[t,j] * y_perm[inv_perm[t*k+j],:]; one thread per 16-byte vector.
+template <typename T>
+__global__ void __launch_bounds__(256) combine_kernel(
+        int T_tokens, int d, int k, const T* __restrict__ y_perm, const int32_t* __restrict__ inv_perm,
+        const float* __restrict__ topk_w, T* __restrict__ out) {
+    constexpr int V = Vec16<T>::N;
+    const int vec_per_row = d / V;
+    const int64_t g = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (g >= static_cast<int64_t>(T_tokens) * vec_per_row) return;
+    const int64_t t = g / vec_per_row;
+    const int c = static_cast<int>(g % vec_per_row) * V;
+    float acc[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = 0.0f;
+    for (int j = 0; j < k; ++j) {
+        const int pos = inv_perm[t * k + j];
+        const float w = topk_w[t * k + j];
+        float y[V];
+        Vec16<T>::load(y_perm + static_cast<int64_t>(pos) * d + c, y);
+#pragma unroll
+        for (int v = 0; v < V; ++v) acc[v] = fmaf(w, y[v], acc[v]);
+    }
+    Vec16<T>::store(out + t * d + c, acc);
+}
+
+}  // namespace
+
+int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_idx, const int32_t* offsets,
+                   int32_t* perm, int32_t* inv_perm, void* x_perm, cudaStream_t s) {
+    const int A = p.T * p.top_k;
+    const int grid = (A + kChunk - 1) / kChunk;
+    if (p.dtype == MONDE_BF16)
+        permute_gather_kernel<__nv_bfloat16><<<grid, kChunk, 0, s>>>(
+            A, p.E, p.top_k, p.d_model, static_cast<const __nv_bfloat16*>(x), topk_idx, offsets, perm,
+            inv_perm, static_cast<__nv_bfloat16*>(x_perm));
+    else
+        permute_gather_kernel<float><<<grid, kChunk, 0, s>>>(
+            A, p.E, p.top_k, p.d_model, static_cast<const float*>(x), topk_idx, offsets, perm, inv_perm,
+            static_cast<float*>(x_perm));
+    return launched();
+}
+
+int launch_combine(const monde_problem& p, const void* y_perm, const int32_t* inv_perm,
+                   const float* topk_w, void* out, cudaStream_t s) {
+    const int V = p.dtype == MONDE_BF16 ? 8 : 4;
+    const int64_t n = static_cast<int64_t>(p.T) * (p.d_model / V);
+    const int grid = static_cast<int>((n + 255) / 256);
+    if (p.dtype == MONDE_BF16)
+        combine_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(
+            p.T, p.d_model, p.top_k, static_cast<const __nv_bfloat16*>(y_perm), inv_perm, topk_w,
+            static_cast<__nv_bfloat16*>(out));
+    else
+        combine_kernel<float><<<grid, 256, 0, s>>>(p.T, p.d_model, p.top_k, static_cast<const float*>(y_perm),
+                                                   inv_perm, topk_w, static_cast<float*>(out));
+    return launched();
+}
+
+}  // namespace monde

@@ -1,0 +1,118 @@
+"""Parity harness: runs the CUDA library through its binding and the CPU oracle on the
+same seeded inputs and compares step by step.
+
+Rules: routing integers, class lists, permutation and x_perm are bit-exact; gate
+weights and probabilities agree to 1e-5 absolute (fp32 softmax); y_perm and out agree
+within max|diff| <= 1e-2 * max|ref| and relative Frobenius error <= 5e-3 for bf16
+problems, and within 1e-5 on both measures for fp32 problems.
+"""
+from __future__ import annotations
+
+from types import SimpleNamespace
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2405_18832_b200 import binding as B
+from paper_2405_18832_b200 import synthetic as S
+
+TOL = {"bf16": (1e-2, 5e-3), "f32": (1e-5, 1e-5)}
+
+
+def widen(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def check_close(name, got64: np.ndarray, ref64: np.ndarray, dtype: str):
+    tol_abs, tol_fro = TOL[dtype]
+    if ref64.size == 0:
+        return 0.0, 0.0
+    scale = np.abs(ref64).max()
+    max_abs = np.abs(got64 - ref64).max()
+    fro = np.linalg.norm(got64 - ref64) / max(np.linalg.norm(ref64), 1e-300)
+    assert np.isfinite(got64).all(), f"{name}: non-finite values"
+    assert max_abs <= tol_abs * scale, f"{name}: max|diff| {max_abs:.3e} > {tol_abs:g} * {scale:.3e}"
+    assert fro <= tol_fro, f"{name}: relative Frobenius error {fro:.3e} > {tol_fro:g}"
+    return max_abs / max(scale, 1e-300), fro
+
+
+def to_device(g, device="cuda"):
+    return {k: (None if v is None else v.to(device)) for k, v in g.items()}
+
+
+def run_gpu(p, dev, want_probs=True):
+    buf = B.LayerBuffers(p, want_probs=want_probs)
+    B.moe_ffn_layer_forward(p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"], buf)
+    B.monde_poll_device_status(buf.ws)
+    return buf
+
+
+def check_routing(p, g, buf):
+    """Bit-exact integer outputs and 1e-5 gate weights against the oracle; returns the oracle's routing."""
+    r = oracle.route(S.as_numpy(g["x"]), S.as_numpy(g["Wg"]), S.as_numpy(g["bg"]),
+                     p.top_k, p.renormalize, p.hot_threshold)
+    np.testing.assert_array_equal(buf.topk_idx.cpu().numpy(), r.topk_idx)
+    np.testing.assert_array_equal(buf.counts.cpu().numpy(), r.counts)
+    np.testing.assert_array_equal(buf.offsets.cpu().numpy(), r.offsets)
+    np.testing.assert_array_equal(buf.cls.cpu().numpy(), r.cls)
+    nh, nc = r.n_hot_cold
+    np.testing.assert_array_equal(buf.n_hot_cold.cpu().numpy(), r.n_hot_cold)
+    np.testing.assert_array_equal(buf.hot_ids.cpu().numpy()[:nh], r.hot_ids[:nh])
+    np.testing.assert_array_equal(buf.cold_ids.cpu().numpy()[:nc], r.cold_ids[:nc])
+    if p.T:
+        assert np.abs(buf.topk_w.cpu().numpy().astype(np.float64) - r.topk_w).max() <= 1e-5
+        if buf.probs is not None:
+            assert np.abs(buf.probs.cpu().numpy().astype(np.float64) - r.probs).max() <= 1e-5
+    pm = oracle.permute(S.as_numpy(g["x"]), r.topk_idx, r.offsets)
+    np.testing.assert_array_equal(buf.perm.cpu().numpy(), pm.perm)
+    np.testing.assert_array_equal(buf.inv_perm.cpu().numpy(), pm.inv_perm)
+    np.testing.assert_array_equal(S.as_numpy(buf.x_perm), pm.x_perm)
+    return r, pm
+
+
+def check_full(w: S.Workload, g=None, dev=None):
+    """Element-by-element parity of every output of the four calls."""
+    p = w.problem
+    g = g if g is not None else S.generate(w)
+    dev = dev if dev is not None else to_device(g)
+    buf = run_gpu(p, dev)
+    r, pm = check_routing(p, g, buf)
+    y_ref = oracle.expert_ffn(pm.x_perm, oracle.experts_of_rows(r.offsets), S.as_numpy(g["W1"]),
+                              S.as_numpy(g["b1"]), S.as_numpy(g["W2"]), S.as_numpy(g["b2"]), p.act)
+    y_err = check_close("y_perm", widen(buf.y_perm), y_ref, p.dtype)
+    out_ref = oracle.combine(y_ref, pm.inv_perm, r.topk_w)
+    out_err = check_close("out", widen(buf.out), out_ref, p.dtype)
+    # combine checked alone: the oracle's combine applied to the device's own y_perm
+    alone = oracle.combine(widen(buf.y_perm), pm.inv_perm, buf.topk_w.cpu().numpy().astype(np.float64))
+    got = widen(buf.out)
+    ulp = 2.0 ** -8 if p.dtype == "bf16" else 2.0 ** -22
+    assert (np.abs(got - alone) <= ulp * np.abs(alone) + 1e-30).all(), "combine: more than one rounding"
+    return SimpleNamespace(buf=buf, route=r, perm=pm, y_err=y_err, out_err=out_err)
+
+
+def check_sampled(w: S.Workload, g, dev, n_tokens=96, buf=None):
+    """Full-size parity: routing in full (bit-exact), expert outputs and the combined
+    output on a deterministic sample of tokens, one oracle FFN row at a time."""
+    p = w.problem
+    buf = buf if buf is not None else run_gpu(p, dev, want_probs=False)
+    r, pm = check_routing(p, g, buf)
+    step = max(1, -(-p.T // n_tokens))
+    tokens = np.arange(0, p.T, step)
+    assign = (tokens[:, None] * p.top_k + np.arange(p.top_k)[None, :]).reshape(-1)
+    rows = pm.inv_perm[assign]
+    experts = r.topk_idx.reshape(-1)[assign]
+    y_ref = np.zeros((rows.size, p.d_model))
+    for e in np.unique(experts):          # one expert's weights on the host at a time
+        sel = np.nonzero(experts == e)[0]
+        W1 = S.as_numpy(dev["W1"][e:e + 1]); W2 = S.as_numpy(dev["W2"][e:e + 1])
+        b1 = S.as_numpy(dev["b1"][e:e + 1]) if dev["b1"] is not None else None
+        b2 = S.as_numpy(dev["b2"][e:e + 1]) if dev["b2"] is not None else None
+        y_ref[sel] = oracle.expert_ffn(pm.x_perm[rows[sel]], np.zeros(sel.size, np.int32), W1, b1, W2, b2, p.act)
+    y_got = widen(buf.y_perm[torch.as_tensor(rows, device=buf.y_perm.device).long()])
+    y_err = check_close("y_perm(sample)", y_got, y_ref, p.dtype)
+    out_ref = oracle.combine(y_ref, np.arange(rows.size, dtype=np.int32), np.ascontiguousarray(r.topk_w[tokens]))
+    out_got = widen(buf.out[torch.as_tensor(tokens, device=buf.out.device).long()])
+    out_err = check_close("out(sample)", out_got, out_ref, p.dtype)
+    assert torch.isfinite(buf.out.float()).all() and torch.isfinite(buf.y_perm.float()).all()
+    return SimpleNamespace(buf=buf, route=r, perm=pm, y_err=y_err, out_err=out_err, n_rows=rows.size)
