@@ -27,7 +27,7 @@
  *  - T == 0 is valid: MONDE_OK, nothing launched.
  *  - Notation (paper Table 1): T = B*S tokens, d_model, d_ff, E experts;
  *    A = T*top_k assignments; an assignment id is a = t*top_k + j.
- *  - Limits: 1 <= top_k <= min(E, 8); E <= 256; bf16 path needs d_model and d_ff
+ *  - Limits: 1 <= top_k <= min(E, 8); E <= 256; T*top_k <= 2^20; bf16 path needs d_model and d_ff
  *    to be multiples of 64; fp32 path needs multiples of 4.
  */
 #ifndef MONDE_H_

@@ -16,7 +16,7 @@ int check_problem(const monde_problem* p) {
     if (p->E > kMaxExperts || p->top_k > kMaxTopK) return MONDE_ERR_UNSUPPORTED;
     const int mult = p->dtype == MONDE_BF16 ? 64 : 4;
     if (p->d_model % mult != 0 || p->d_ff % mult != 0) return MONDE_ERR_UNSUPPORTED;
-    if (static_cast<int64_t>(p->T) * p->top_k > (1ll << 30)) return MONDE_ERR_UNSUPPORTED;
+    if (static_cast<int64_t>(p->T) * p->top_k > kMaxAssignments) return MONDE_ERR_UNSUPPORTED;
     return MONDE_OK;
 }
 
@@ -161,8 +161,8 @@ int monde_poll_device_status(void* ws, void* stream, int32_t* site) {
         return MONDE_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return MONDE_ERR_CUDA;
     if (site != nullptr) *site = word[1];
-    if (word[0] != 0) {
-        if (cudaMemsetAsync(static_cast<char*>(ws) + WsLayout::kStatus, 0, sizeof word, s) != cudaSuccess)
+    if (word[0] != 0) {   // a kernel gave up: its counters may be mid-way, so clear the whole header
+        if (cudaMemsetAsync(ws, 0, WsLayout::kHidden, s) != cudaSuccess)
             return MONDE_ERR_CUDA;
         if (cudaStreamSynchronize(s) != cudaSuccess) return MONDE_ERR_CUDA;
     }

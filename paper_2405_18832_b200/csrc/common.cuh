@@ -25,6 +25,11 @@ struct WsLayout {
     size_t hidden_bytes;
     size_t total;
 };
+// The header (first kHidden bytes) holds everything that must be zero between calls: the
+// status word, the CTA ticket (kCounters) and one int32 per token tile that counts finished
+// first-layer units (kTiles).  A <= kMaxAssignments keeps the token-tile counters inside it.
+constexpr int64_t kMaxAssignments = 1 << 20;
+static_assert(4 * (kMaxAssignments / 64 + 2 * 256 + 64) <= 112 * 1024, "token-tile counters overflow the header");
 
 inline size_t elem_bytes(int dtype) { return dtype == MONDE_BF16 ? 2 : 4; }
 

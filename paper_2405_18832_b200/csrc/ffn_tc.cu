@@ -1,21 +1,29 @@
-// bf16 expert linear layers on the 5th-generation tensor cores (tcgen05, accumulators in
-// tensor memory), operands staged in shared memory by TMA.
+// bf16 expert FFN on the 5th-generation tensor cores (tcgen05, accumulators in tensor
+// memory), operands staged in shared memory by TMA; one persistent launch runs both
+// linear layers of every activated expert, hot and cold.
 //
 // Paper: Section 3.1 describes an expert computation as C = A x B with A the routed
 // tokens (small height for cold experts) and B the expert parameters (width d_model or
 // d_ff); Section 2.2 separates hot experts (many tokens) from cold, memory-bound ones;
-// Section 3.4 names the gemm and gemm+activation kernels.  Here every expert GEMM is
-// issued "weights as rows": the 128-row MMA dimension holds 128 output features of the
-// expert's weight matrix and the MMA N dimension holds the tokens, so an expert with m
-// tokens costs one pass over its weights with N = m rounded up to 16.  The two classes
-// are two instantiations of the same kernel:
-//   cold: token tile <= 64, 8-stage ring of 24 KB stages -> a deep queue of weight bytes
-//         in flight per SM; the tensor core is idle most of the time and HBM sets the pace;
-//   hot : token tile <= 256 (a full-rate 128 x 256 MMA), 4-stage ring of 48 KB stages.
+// Section 3.3 runs the two classes side by side on the hardware that suits each;
+// Section 3.4 names the gemm and gemm+activation kernels.
+//
+// Every expert GEMM is issued "weights as rows": the 128-row MMA dimension holds 128
+// output features of the expert's weight matrix and the MMA N dimension holds the tokens,
+// so an expert with m tokens costs one pass over its weights with N = m rounded up to 16.
+// The class chosen by the router selects the tiling of a work unit:
+//   hot : token tile <= 256 (a full-rate 128 x 256 MMA), 4-stage ring of 48 KB stages;
+//   cold: token tile <= 64, 8-stage ring of 24 KB stages -> a deep queue of weight bytes in
+//         flight per SM; the tensor core idles most of the time and HBM sets the pace.
+// Work units (expert, 128-feature tile, token tile) are ordered hot-first-layer,
+// hot-second-layer, cold-first-layer, cold-second-layer and dealt round-robin to one
+// persistent CTA per SM.  A second-layer unit needs the hidden rows of its token tile,
+// which are produced by first-layer units earlier in the same order: per-token-tile
+// counters in the workspace carry that dependency, and the TMA producer streams the
+// unit's weights while it waits, so weight traffic never stalls at the layer boundary.
 // Warp roles: warp 0 issues TMA, warp 1 issues MMAs and owns the TMEM allocation, warps
-// 2-5 drain the accumulator (bias + activation fused) while the next tile's MMAs run into
-// the second accumulator buffer.  CTAs are persistent and walk a device-built list of
-// (expert, feature tile, token tile) units, so counts never travel to the host.
+// 2-5 drain the accumulator (bias + activation fused) while the next unit's MMAs run into
+// the second accumulator buffer.  Counts never travel to the host.
 #include <cuda.h>
 
 #include <mutex>
@@ -33,19 +41,33 @@ constexpr int kThreads = 192;
 constexpr int kBlockK = 64;           // K elements per stage: one 128-byte swizzle row
 constexpr int kTileRows = 128;        // output features per unit = MMA M
 constexpr int kABytes = kTileRows * 128;
+constexpr int kMaxStages = 8;
+constexpr int kHotTokTile = 256, kHotStages = 4;     // 4 x (16 KB + 32 KB)
+constexpr int kColdTokTile = 64, kColdStages = 8;    // 8 x (16 KB +  8 KB)
+constexpr int kTileBytes = 192 * 1024;
+constexpr int kNumBars = 2 * kMaxStages + 4;
+constexpr int kTableInts = 6 * (kMaxExperts + 1);
+constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kTableInts * 4;
+constexpr int kTmemCols = 512;        // two accumulator buffers of 256 fp32 columns
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
 
-enum WaitSite { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4 };
+enum WaitSite { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4,
+                kSiteHiddenReady = 5, kSiteDrain = 6 };
 
-template <int kTokTile, int kStages>
-struct Cfg {
-    static constexpr int kBBytes = kTokTile * 128;
-    static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kTileBytes = kStages * kStageBytes;
-    static constexpr int kNumBars = 2 * kStages + 4;
-    static constexpr int kTableInts = 6 * (kMaxExperts + 1);
-    static constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kTableInts * 4;
-    static constexpr int kTmemCols = 2 * kTokTile < 32 ? 32 : 2 * kTokTile;   // power of two for 64 / 256
+struct FfnParams {
+    int d_model, d_ff, act;
+    const __nv_bfloat16* b1;
+    const __nv_bfloat16* b2;
+    __nv_bfloat16* h;
+    __nv_bfloat16* y;
+    const int32_t* counts;
+    const int32_t* offsets;
+    const int32_t* hot_ids;
+    const int32_t* cold_ids;
+    const int32_t* n_hot_cold;
+    int32_t* status;       // {status, site}
+    int32_t* ticket;       // CTAs that have finished
+    int32_t* ready;        // per token tile: first-layer units finished (x4, one per epilogue warp)
 };
 
 struct Unit {
@@ -54,26 +76,47 @@ struct Unit {
     int rows;     // valid token rows in the tile
     int nt;       // rows rounded up to a multiple of 16 (MMA N)
     int n0;       // first output feature of the tile
+    int layer;    // 0: h = act(x W1^T + b1), 1: y = h W2^T + b2
+    int cold;     // class: selects the stage geometry
+    int ready_idx;  // token-tile index into the dependency counters
 };
 
+// Per-CTA copy of the unit list in shared memory.  Entries 0..n_hot-1 are the hot experts,
+// n_hot..n_hot+n_cold-1 the cold ones; tt_prefix is the exclusive prefix of token tiles.
 struct UnitTable {
-    int* prefix;  // [n+1] exclusive prefix of units per listed expert
+    int* tt_prefix;   // [n+1]
     int* e;
     int* off;
     int* m;
-    int* tt;      // token tiles
-    int* per;     // tokens per tile (multiple of 16)
-    __device__ __forceinline__ Unit decode(int u, int& cursor) const {
-        while (u >= prefix[cursor + 1]) ++cursor;
-        const int local = u - prefix[cursor];
-        const int tok = local % tt[cursor];
+    int* tt;          // token tiles of this expert
+    int* per;         // tokens per tile (multiple of 16)
+    int n_hot, n_all, nt1, nt2;      // 128-feature tiles of layer 1 (d_ff) and layer 2 (d_model)
+    int seg[5];                      // unit index where each (class, layer) segment starts
+
+    __device__ __forceinline__ Unit decode(int u) const {
+        int sgm = 0;
+        while (u >= seg[sgm + 1]) ++sgm;
         Unit r;
-        r.e = e[cursor];
-        r.n0 = (local / tt[cursor]) * kTileRows;
-        const int r_in_e = tok * per[cursor];
-        r.rows = min(per[cursor], m[cursor] - r_in_e);
+        r.cold = sgm >> 1;
+        r.layer = sgm & 1;
+        const int ntl = r.layer ? nt2 : nt1;
+        const int lo_entry = r.cold ? n_hot : 0;
+        const int tt_base = tt_prefix[lo_entry];
+        const int v = u - seg[sgm];
+        int lo = lo_entry, hi = (r.cold ? n_all : n_hot) - 1;      // largest entry with block start <= v
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if ((tt_prefix[mid] - tt_base) * ntl <= v) lo = mid; else hi = mid - 1;
+        }
+        const int local = v - (tt_prefix[lo] - tt_base) * ntl;
+        const int tok = local % tt[lo];
+        r.e = e[lo];
+        r.n0 = (local / tt[lo]) * kTileRows;
+        const int r_in_e = tok * per[lo];
+        r.rows = min(per[lo], m[lo] - r_in_e);
         r.nt = (r.rows + 15) & ~15;
-        r.row0 = off[cursor] + r_in_e;
+        r.row0 = off[lo] + r_in_e;
+        r.ready_idx = tt_prefix[lo] + tok;
         return r;
     }
 };
@@ -83,22 +126,24 @@ __device__ __forceinline__ void report_timeout(int32_t* status, volatile int* ab
     if (atomicCAS(status, 0, MONDE_ERR_TIMEOUT) == 0) status[1] = site;
 }
 
-// Out[row, n] = act?(bias[e, n] + sum_k In[row, k] * W[e, n, k]) for the rows of the listed experts.
-template <int kTokTile, int kStages>
-__global__ void __launch_bounds__(kThreads, 1) expert_gemm_kernel(
-        const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_in,
-        int K, int N, int act, const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ out,
-        const int32_t* __restrict__ counts, const int32_t* __restrict__ offsets,
-        const int32_t* __restrict__ ids, const int32_t* __restrict__ n_ids, int32_t* status) {
-    using C = Cfg<kTokTile, kStages>;
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
+        const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
+        const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_h, const FfnParams P) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kTileBytes);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C::kNumBars);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTileBytes);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* tab = reinterpret_cast<int*>(tmem_slot + 16);
     UnitTable ut;
-    ut.prefix = tab;
+    ut.tt_prefix = tab;
     ut.e = tab + (kMaxExperts + 1);
     ut.off = ut.e + (kMaxExperts + 1);
     ut.m = ut.off + (kMaxExperts + 1);
@@ -106,43 +151,45 @@ __global__ void __launch_bounds__(kThreads, 1) expert_gemm_kernel(
     ut.per = ut.tt + (kMaxExperts + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n_list = min(*n_ids, kMaxExperts);
-    const int n_tiles = (N + kTileRows - 1) / kTileRows;
-    const int k_blocks = K / kBlockK;
+    ut.n_hot = min(P.n_hot_cold[0], kMaxExperts);
+    ut.n_all = min(ut.n_hot + P.n_hot_cold[1], kMaxExperts);
+    ut.nt1 = (P.d_ff + kTileRows - 1) / kTileRows;
+    ut.nt2 = (P.d_model + kTileRows - 1) / kTileRows;
 
     // ---- set-up: unit table, barriers, tensor memory --------------------------------
-    for (int i = tid; i < n_list; i += kThreads) {
-        const int e = ids[i];
-        const int m = counts[e];
-        const int tt = (m + kTokTile - 1) / kTokTile;
-        const int per = tt > 0 ? (((m + tt - 1) / tt + 15) & ~15) : 16;
+    for (int i = tid; i < ut.n_all; i += kThreads) {
+        const bool cold = i >= ut.n_hot;
+        const int e = cold ? P.cold_ids[i - ut.n_hot] : P.hot_ids[i];
+        const int tile = cold ? kColdTokTile : kHotTokTile;
+        const int m = P.counts[e];
+        const int tt = max(1, (m + tile - 1) / tile);
         ut.e[i] = e;
-        ut.off[i] = offsets[e];
+        ut.off[i] = P.offsets[e];
         ut.m[i] = m;
-        ut.tt[i] = tt > 0 ? tt : 1;
-        ut.per[i] = per;
-        ut.prefix[i + 1] = tt * n_tiles;
+        ut.tt[i] = tt;
+        ut.per[i] = ((m + tt - 1) / tt + 15) & ~15;
+        ut.tt_prefix[i + 1] = tt;
     }
     if (tid == 0) {
-        ut.prefix[0] = 0;
+        ut.tt_prefix[0] = 0;
         *abort_flag = 0;
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&bars[s]), 1);             // full: producer's expect_tx arrival
-            mbar_init(smem_u32(&bars[kStages + s]), 1);   // empty: one tcgen05.commit
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&bars[s]), 1);               // full: producer's expect_tx arrival
+            mbar_init(smem_u32(&bars[kMaxStages + s]), 1);  // empty: one tcgen05.commit
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&bars[2 * kStages + b]), 1);       // accumulator full: one commit
-            mbar_init(smem_u32(&bars[2 * kStages + 2 + b]), 4);   // accumulator drained: 4 epilogue warps
+            mbar_init(smem_u32(&bars[2 * kMaxStages + b]), 1);       // accumulator full: one commit
+            mbar_init(smem_u32(&bars[2 * kMaxStages + 2 + b]), 4);   // accumulator drained: 4 epilogue warps
         }
         fence_barrier_init();
     }
     __syncthreads();
-    if (warp == 0) {   // inclusive scan of the per-expert unit counts, 8 entries per lane
+    if (warp == 0) {   // inclusive scan of the per-expert token-tile counts, 8 entries per lane
         int v[8], sum = 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int idx = lane * 8 + i;
-            v[i] = idx < n_list ? ut.prefix[idx + 1] : 0;
+            v[i] = idx < ut.n_all ? ut.tt_prefix[idx + 1] : 0;
             sum += v[i];
         }
         int inc = sum;
@@ -156,101 +203,158 @@ __global__ void __launch_bounds__(kThreads, 1) expert_gemm_kernel(
         for (int i = 0; i < 8; ++i) {
             const int idx = lane * 8 + i;
             run += v[i];
-            if (idx < n_list) ut.prefix[idx + 1] = run;
+            if (idx < ut.n_all) ut.tt_prefix[idx + 1] = run;
         }
     } else if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), C::kTmemCols);
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const int total_units = ut.prefix[n_list];
+    const int tt_hot = ut.tt_prefix[ut.n_hot], tt_all = ut.tt_prefix[ut.n_all];
+    ut.seg[0] = 0;
+    ut.seg[1] = tt_hot * ut.nt1;
+    ut.seg[2] = ut.seg[1] + tt_hot * ut.nt2;
+    ut.seg[3] = ut.seg[2] + (tt_all - tt_hot) * ut.nt1;
+    ut.seg[4] = ut.seg[3] + (tt_all - tt_hot) * ut.nt2;
+    const int total_units = ut.seg[4];
     const uint32_t tiles_u32 = smem_u32(smem);
+    const int ready_target = 4 * ut.nt1;
 
     if (warp == 0) {
         // ---- TMA producer ------------------------------------------------------------
         if (lane == 0) {
-            prefetch_tensormap(&map_w);
-            prefetch_tensormap(&map_in);
+            prefetch_tensormap(&map_w1);
+            prefetch_tensormap(&map_w2);
+            prefetch_tensormap(&map_x);
+            prefetch_tensormap(&map_h);
             const uint64_t pol_w = policy_evict_first();   // weights are read once
             const uint64_t pol_x = policy_evict_last();    // token tiles are re-read by every feature tile
-            int stage = 0, cursor = 0;
-            uint32_t phase = 0;
+            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = kABytes + kHotTokTile * 128;
+            uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
             bool ok = true;
             for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
-                const Unit un = ut.decode(u, cursor);
+                const Unit un = ut.decode(u);
+                if (un.cold != cls) {
+                    // geometry switch: every stage filled so far must have been consumed
+                    for (int s = 0; ok && s < stages; ++s)
+                        if (!mbar_wait(smem_u32(&bars[kMaxStages + s]), ((fill_bits >> s) & 1u) ^ 1u, abort_flag,
+                                       kWaitLimitNs)) {
+                            report_timeout(P.status, abort_flag, kSiteDrain);
+                            ok = false;
+                        }
+                    if (!ok) break;
+                    cls = un.cold;
+                    stages = cls ? kColdStages : kHotStages;
+                    stage_bytes = kABytes + (cls ? kColdTokTile : kHotTokTile) * 128;
+                    stage = 0;
+                }
+                const CUtensorMap* mw = un.layer ? &map_w2 : &map_w1;
+                const CUtensorMap* mi = un.layer ? &map_h : &map_x;
+                const int K = un.layer ? P.d_ff : P.d_model;
+                const int N = un.layer ? P.d_model : P.d_ff;
+                const int k_blocks = K / kBlockK;
                 for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!mbar_wait(smem_u32(&bars[kStages + stage]), phase ^ 1u, abort_flag, kWaitLimitNs)) {
-                        report_timeout(status, abort_flag, kSiteProducerEmpty);
+                    if (!mbar_wait(smem_u32(&bars[kMaxStages + stage]), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag,
+                                   kWaitLimitNs)) {
+                        report_timeout(P.status, abort_flag, kSiteProducerEmpty);
                         ok = false;
                         break;
                     }
                     const uint32_t full = smem_u32(&bars[stage]);
-                    const uint32_t a_dst = tiles_u32 + stage * C::kStageBytes;
+                    const uint32_t a_dst = tiles_u32 + stage * stage_bytes;
                     mbar_arrive_expect_tx(full, kABytes + un.nt * 128);
-                    tma_load_2d(a_dst, &map_w, full, kb * kBlockK, un.e * N + un.n0, pol_w);
+                    tma_load_2d(a_dst, mw, full, kb * kBlockK, un.e * N + un.n0, pol_w);
+                    if (kb == 0 && un.layer == 1) {
+                        // the hidden rows of this token tile must be complete; weights already stream
+                        const int32_t* flag = P.ready + un.ready_idx;
+                        if (ld_acquire(flag) < ready_target) {
+                            const uint64_t t0 = global_timer_ns();
+                            while (ld_acquire(flag) < ready_target) {
+                                if (*abort_flag != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
+                                    report_timeout(P.status, abort_flag, kSiteHiddenReady);
+                                    ok = false;
+                                    break;
+                                }
+                            }
+                            if (!ok) break;
+                        }
+                        fence_proxy_async_all();
+                    }
                     for (int j = 0; j < un.nt; j += 16)
-                        tma_load_2d(a_dst + kABytes + j * 128, &map_in, full, kb * kBlockK, un.row0 + j, pol_x);
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                        tma_load_2d(a_dst + kABytes + j * 128, mi, full, kb * kBlockK, un.row0 + j, pol_x);
+                    fill_bits ^= 1u << stage;
+                    if (++stage == stages) stage = 0;
                 }
             }
         }
     } else if (warp == 1) {
         // ---- MMA issuer --------------------------------------------------------------
         if (lane == 0) {
-            int stage = 0, cursor = 0, it = 0;
-            uint32_t phase = 0;
+            int stage = 0, it = 0, cls = -1, stages = kHotStages, stage_bytes = kABytes + kHotTokTile * 128;
+            uint32_t use_bits = 0;      // bit s: parity of the number of uses of stage s
             bool ok = true;
             for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x, ++it) {
-                const Unit un = ut.decode(u, cursor);
+                const Unit un = ut.decode(u);
+                if (un.cold != cls) {
+                    cls = un.cold;
+                    stages = cls ? kColdStages : kHotStages;
+                    stage_bytes = kABytes + (cls ? kColdTokTile : kHotTokTile) * 128;
+                    stage = 0;
+                }
                 const int b = it & 1;
                 const uint32_t tphase = (it >> 1) & 1;
-                if (!mbar_wait(smem_u32(&bars[2 * kStages + 2 + b]), tphase ^ 1u, abort_flag, kWaitLimitNs)) {
-                    report_timeout(status, abort_flag, kSiteMmaTmemEmpty);
+                if (!mbar_wait(smem_u32(&bars[2 * kMaxStages + 2 + b]), tphase ^ 1u, abort_flag, kWaitLimitNs)) {
+                    report_timeout(P.status, abort_flag, kSiteMmaTmemEmpty);
                     break;
                 }
                 tc_fence_after_sync();
                 const uint32_t idesc = idesc_bf16_m128(un.nt);
-                const uint32_t d_tmem = tmem_base + b * kTokTile;
+                const uint32_t d_tmem = tmem_base + b * 256;
+                const int k_blocks = (un.layer ? P.d_ff : P.d_model) / kBlockK;
                 for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!mbar_wait(smem_u32(&bars[stage]), phase, abort_flag, kWaitLimitNs)) {
-                        report_timeout(status, abort_flag, kSiteMmaFull);
+                    if (!mbar_wait(smem_u32(&bars[stage]), (use_bits >> stage) & 1u, abort_flag, kWaitLimitNs)) {
+                        report_timeout(P.status, abort_flag, kSiteMmaFull);
                         ok = false;
                         break;
                     }
                     tc_fence_after_sync();
-                    const uint32_t a_addr = tiles_u32 + stage * C::kStageBytes;
+                    const uint32_t a_addr = tiles_u32 + stage * stage_bytes;
                     const uint64_t a_desc = smem_desc_sw128(a_addr);
                     const uint64_t b_desc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
                     for (int k4 = 0; k4 < kBlockK / 16; ++k4)
                         umma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kb | k4) != 0);
-                    umma_commit(smem_u32(&bars[kStages + stage]));   // stage reusable once these MMAs finish
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    umma_commit(smem_u32(&bars[kMaxStages + stage]));   // stage reusable once these MMAs finish
+                    use_bits ^= 1u << stage;
+                    if (++stage == stages) stage = 0;
                 }
-                if (ok) umma_commit(smem_u32(&bars[2 * kStages + b]));   // accumulator complete
+                if (ok) umma_commit(smem_u32(&bars[2 * kMaxStages + b]));   // accumulator complete
             }
         }
     } else {
         // ---- epilogue: TMEM -> registers -> bias, activation -> global ----------------
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
-        int cursor = 0, it = 0;
+        int it = 0;
         for (int u = blockIdx.x; u < total_units; u += gridDim.x, ++it) {
-            const Unit un = ut.decode(u, cursor);
+            const Unit un = ut.decode(u);
             const int b = it & 1;
             const uint32_t tphase = (it >> 1) & 1;
-            if (!mbar_wait(smem_u32(&bars[2 * kStages + b]), tphase, abort_flag, kWaitLimitNs)) {
-                report_timeout(status, abort_flag, kSiteEpilogueTmemFull);
+            if (!mbar_wait(smem_u32(&bars[2 * kMaxStages + b]), tphase, abort_flag, kWaitLimitNs)) {
+                report_timeout(P.status, abort_flag, kSiteEpilogueTmemFull);
                 break;
             }
             tc_fence_after_sync();
+            const int N = un.layer ? P.d_model : P.d_ff;
+            const int act = un.layer ? -1 : P.act;
+            const __nv_bfloat16* bias = un.layer ? P.b2 : P.b1;
             const int n = un.n0 + q * 32 + lane;
             const bool n_ok = n < N;
             const float bias_v = (bias != nullptr && n_ok) ? __bfloat162float(bias[static_cast<int64_t>(un.e) * N + n]) : 0.0f;
-            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * kTokTile;
-            __nv_bfloat16* dst = out + static_cast<int64_t>(un.row0) * N + n;
+            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 256;
+            __nv_bfloat16* dst = (un.layer ? P.y : P.h) + static_cast<int64_t>(un.row0) * N + n;
             for (int c0 = 0; c0 < un.nt; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld_16(t_addr + c0, v);
@@ -267,8 +371,17 @@ __global__ void __launch_bounds__(kThreads, 1) expert_gemm_kernel(
                 }
             }
             tc_fence_before_sync();
+            if (un.layer == 0) {
+                // publish the hidden rows: stores visible device-wide (and to the async proxy
+                // that will read them through TMA) before the counter moves
+                __threadfence();
+                fence_proxy_async_all();
+            }
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars[2 * kStages + 2 + b]));
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&bars[2 * kMaxStages + 2 + b]));
+                if (un.layer == 0) atomicAdd(P.ready + un.ready_idx, 1);
+            }
         }
     }
 
@@ -277,7 +390,20 @@ __global__ void __launch_bounds__(kThreads, 1) expert_gemm_kernel(
     __syncthreads();
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, C::kTmemCols);
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    // The last CTA to finish leaves the dependency counters at zero for the next call.
+    if (warp == 2) {
+        int last = 0;
+        if (lane == 0) {
+            __threadfence();
+            last = atomicAdd(P.ticket, 1) == static_cast<int>(gridDim.x) - 1;
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+            for (int i = lane; i < tt_all; i += 32) P.ready[i] = 0;
+            if (lane == 0) *P.ticket = 0;
+        }
     }
 }
 
@@ -322,50 +448,43 @@ int sm_count() {
     return n;
 }
 
-template <int kTokTile, int kStages>
-int launch_one(int E, int rows_total, int K, int N, int act, const void* in, const void* W, const void* bias,
-               void* out, const int32_t* counts, const int32_t* offsets, const int32_t* ids,
-               const int32_t* n_ids, int32_t* status, cudaStream_t s) {
-    using C = Cfg<kTokTile, kStages>;
-    auto kernel = expert_gemm_kernel<kTokTile, kStages>;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    });
-    if (attr_err != cudaSuccess) return MONDE_ERR_CUDA;
-    CUtensorMap map_w, map_in;
-    if (!make_map(&map_w, W, static_cast<uint64_t>(E) * N, K, kTileRows)) return MONDE_ERR_CUDA;
-    if (!make_map(&map_in, in, rows_total, K, 16)) return MONDE_ERR_CUDA;
-    kernel<<<sm_count(), kThreads, C::kSmemBytes, s>>>(
-        map_w, map_in, K, N, act, static_cast<const __nv_bfloat16*>(bias), static_cast<__nv_bfloat16*>(out), counts,
-        offsets, ids, n_ids, status);
-    return launched();
-}
-
 }  // namespace
 
 int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, const void* b1,
                     const void* W2, const void* b2, const int32_t* counts, const int32_t* offsets,
                     const int32_t* hot_ids, const int32_t* cold_ids, const int32_t* n_hot_cold,
                     void* y_perm, void* ws, cudaStream_t s) {
-    void* h = static_cast<char*>(ws) + WsLayout::kHidden;
-    int32_t* status = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + WsLayout::kStatus);
-    const int A = p.T * p.top_k;
-    int st;
-    // cold class: weight-streaming configuration
-    st = launch_one<64, 8>(p.E, A, p.d_model, p.d_ff, p.act, x_perm, W1, b1, h, counts, offsets, cold_ids,
-                           n_hot_cold + 1, status, s);
-    if (st != MONDE_OK) return st;
-    // hot class: wide token tiles
-    st = launch_one<256, 4>(p.E, A, p.d_model, p.d_ff, p.act, x_perm, W1, b1, h, counts, offsets, hot_ids,
-                            n_hot_cold, status, s);
-    if (st != MONDE_OK) return st;
-    st = launch_one<64, 8>(p.E, A, p.d_ff, p.d_model, -1, h, W2, b2, y_perm, counts, offsets, cold_ids,
-                           n_hot_cold + 1, status, s);
-    if (st != MONDE_OK) return st;
-    return launch_one<256, 4>(p.E, A, p.d_ff, p.d_model, -1, h, W2, b2, y_perm, counts, offsets, hot_ids,
-                              n_hot_cold, status, s);
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(expert_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return MONDE_ERR_CUDA;
+    char* base = static_cast<char*>(ws);
+    const uint64_t A = static_cast<uint64_t>(p.T) * p.top_k;
+    FfnParams P;
+    P.d_model = p.d_model;
+    P.d_ff = p.d_ff;
+    P.act = p.act;
+    P.b1 = static_cast<const __nv_bfloat16*>(b1);
+    P.b2 = static_cast<const __nv_bfloat16*>(b2);
+    P.h = reinterpret_cast<__nv_bfloat16*>(base + WsLayout::kHidden);
+    P.y = static_cast<__nv_bfloat16*>(y_perm);
+    P.counts = counts;
+    P.offsets = offsets;
+    P.hot_ids = hot_ids;
+    P.cold_ids = cold_ids;
+    P.n_hot_cold = n_hot_cold;
+    P.status = reinterpret_cast<int32_t*>(base + WsLayout::kStatus);
+    P.ticket = reinterpret_cast<int32_t*>(base + WsLayout::kCounters);
+    P.ready = reinterpret_cast<int32_t*>(base + WsLayout::kTiles);
+    CUtensorMap map_w1, map_w2, map_x, map_h;
+    if (!make_map(&map_w1, W1, static_cast<uint64_t>(p.E) * p.d_ff, p.d_model, kTileRows)) return MONDE_ERR_CUDA;
+    if (!make_map(&map_w2, W2, static_cast<uint64_t>(p.E) * p.d_model, p.d_ff, kTileRows)) return MONDE_ERR_CUDA;
+    if (!make_map(&map_x, x_perm, A, p.d_model, 16)) return MONDE_ERR_CUDA;
+    if (!make_map(&map_h, P.h, A, p.d_ff, 16)) return MONDE_ERR_CUDA;
+    expert_ffn_kernel<<<sm_count(), kThreads, kSmemBytes, s>>>(map_w1, map_w2, map_x, map_h, P);
+    return launched();
 }
 
 }  // namespace monde

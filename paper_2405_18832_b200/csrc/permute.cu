@@ -8,48 +8,42 @@ namespace monde {
 
 namespace {
 
-constexpr int kChunk = 128;          // assignments per CTA
-constexpr int kWarps = kChunk / 32;
+constexpr int kChunk = 32;           // assignments per CTA: one warp ranks them
+constexpr int kThreads = 128;        // all four warps copy rows
 
 // CTA c owns assignments [c*kChunk, (c+1)*kChunk).  The number of earlier assignments to
 // each expert is recounted from topk_idx (at most A integers, L2-resident), which keeps
 // the kernel single-pass and free of inter-CTA ordering.
 template <typename T>
-__global__ void __launch_bounds__(kChunk) permute_gather_kernel(
+__global__ void __launch_bounds__(kThreads) permute_gather_kernel(
         int A, int E, int k, int d, const T* __restrict__ x, const int32_t* __restrict__ topk_idx,
         const int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
         T* __restrict__ x_perm) {
-    __shared__ int before[kMaxExperts];              // assignments to e in earlier chunks
-    __shared__ int warp_cnt[kWarps][kMaxExperts];    // assignments to e per warp of this chunk
+    __shared__ int before[kMaxExperts];   // assignments to e in earlier chunks
     __shared__ int row_pos[kChunk];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int first = blockIdx.x * kChunk;
-    for (int e = tid; e < kMaxExperts; e += kChunk) {
-        before[e] = 0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) warp_cnt[w][e] = 0;
-    }
+    for (int e = tid; e < kMaxExperts; e += kThreads) before[e] = 0;
     __syncthreads();
-    for (int a = tid; a < first; a += kChunk) atomicAdd(&before[topk_idx[a]], 1);
-    const int a = first + tid;
-    const int e = a < A ? topk_idx[a] : -1;
-    const unsigned same = __match_any_sync(0xffffffffu, e);
-    const int rank_in_warp = __popc(same & ((1u << lane) - 1u));
-    if (e >= 0 && rank_in_warp == 0) warp_cnt[warp][e] = __popc(same);
+    for (int a = tid; a < first; a += kThreads) atomicAdd(&before[topk_idx[a]], 1);
     __syncthreads();
-    int pos = -1;
-    if (e >= 0) {
-        pos = offsets[e] + before[e] + rank_in_warp;
-        for (int w = 0; w < warp; ++w) pos += warp_cnt[w][e];
-        perm[pos] = a;
-        inv_perm[a] = pos;
+    if (warp == 0) {
+        const int a = first + lane;
+        const int e = a < A ? topk_idx[a] : -1;
+        const unsigned same = __match_any_sync(0xffffffffu, e);
+        int pos = -1;
+        if (e >= 0) {
+            pos = offsets[e] + before[e] + __popc(same & ((1u << lane) - 1u));
+            perm[pos] = a;
+            inv_perm[a] = pos;
+        }
+        row_pos[lane] = pos;
     }
-    row_pos[tid] = pos;
     __syncthreads();
     // Row gather: each warp copies whole rows with 16-byte accesses.
     constexpr int V = Vec16<T>::N;
     const int vec_per_row = d / V;
-    for (int r = warp; r < kChunk; r += kWarps) {
+    for (int r = warp; r < kChunk; r += kThreads / 32) {
         const int p = row_pos[r];
         if (p < 0) break;
         const uint4* src = reinterpret_cast<const uint4*>(x + static_cast<int64_t>((first + r) / k) * d);
@@ -90,11 +84,11 @@ int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_id
     const int A = p.T * p.top_k;
     const int grid = (A + kChunk - 1) / kChunk;
     if (p.dtype == MONDE_BF16)
-        permute_gather_kernel<__nv_bfloat16><<<grid, kChunk, 0, s>>>(
+        permute_gather_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(
             A, p.E, p.top_k, p.d_model, static_cast<const __nv_bfloat16*>(x), topk_idx, offsets, perm,
             inv_perm, static_cast<__nv_bfloat16*>(x_perm));
     else
-        permute_gather_kernel<float><<<grid, kChunk, 0, s>>>(
+        permute_gather_kernel<float><<<grid, kThreads, 0, s>>>(
             A, p.E, p.top_k, p.d_model, static_cast<const float*>(x), topk_idx, offsets, perm, inv_perm,
             static_cast<float*>(x_perm));
     return launched();

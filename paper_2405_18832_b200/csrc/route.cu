@@ -123,6 +123,89 @@ __global__ void __launch_bounds__(128) route_warp_per_token_kernel(
     softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs);
 }
 
+
+// ---- bf16 gate on the warp-level tensor-core path -------------------------------------
+// CTA = 16 tokens x all experts; each of the 4 warps owns a contiguous quarter of the
+// (padded) expert range as 8-wide MMA column tiles.  Fragments are loaded straight from
+// global memory with 16-byte loads: lane (g, t) reads 8 consecutive k of row g, which
+// feeds the k-slots of two m16n8k16 MMAs.  The k index inside an MMA is permuted the same
+// way for both operands, which leaves every dot product unchanged.  Products of two bf16
+// values are exact in fp32 and accumulation is fp32, so logits keep fp32 accuracy.
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int kTilesPerWarp>   // 8-expert column tiles per warp: padded E = 32 * kTilesPerWarp
+__global__ void __launch_bounds__(128) route_mma_kernel(
+        int T_tokens, int d, int E, int k, int renorm, const __nv_bfloat16* __restrict__ x,
+        const __nv_bfloat16* __restrict__ Wg, const float* __restrict__ bg, int32_t* __restrict__ topk_idx,
+        float* __restrict__ topk_w, float* __restrict__ probs) {
+    constexpr int kEPad = 32 * kTilesPerWarp;
+    __shared__ float s_logit[16][kEPad + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t4 = lane & 3;
+    const int tok0 = blockIdx.x * 16;
+    const int r0 = min(tok0 + g, T_tokens - 1), r1 = min(tok0 + g + 8, T_tokens - 1);
+    const uint4* xa = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(r0) * d) + t4;
+    const uint4* xb = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(r1) * d) + t4;
+    const uint4* wp[kTilesPerWarp];
+#pragma unroll
+    for (int j = 0; j < kTilesPerWarp; ++j) {
+        const int e = min(warp * (8 * kTilesPerWarp) + j * 8 + g, E - 1);
+        wp[j] = reinterpret_cast<const uint4*>(Wg + static_cast<int64_t>(e) * d) + t4;
+    }
+    float acc[kTilesPerWarp][4];
+#pragma unroll
+    for (int j = 0; j < kTilesPerWarp; ++j)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[j][i] = 0.0f;
+    const int steps = d / 32;               // 32 k per step: 4 lanes x 8 elements
+#pragma unroll 2
+    for (int s = 0; s < steps; ++s) {
+        const uint4 a = xa[s * 4], b = xb[s * 4];
+#pragma unroll
+        for (int j = 0; j < kTilesPerWarp; ++j) {
+            const uint4 w = wp[j][s * 4];
+            mma_bf16_16816(acc[j], a.x, b.x, a.y, b.y, w.x, w.y);
+            mma_bf16_16816(acc[j], a.z, b.z, a.w, b.w, w.z, w.w);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < kTilesPerWarp; ++j) {
+        const int e = warp * (8 * kTilesPerWarp) + j * 8 + t4 * 2;
+        const float b0 = (bg != nullptr && e < E) ? bg[e] : 0.0f;
+        const float b1 = (bg != nullptr && e + 1 < E) ? bg[e + 1] : 0.0f;
+        s_logit[g][e] = acc[j][0] + b0;
+        s_logit[g][e + 1] = acc[j][1] + b1;
+        s_logit[g + 8][e] = acc[j][2] + b0;
+        s_logit[g + 8][e + 1] = acc[j][3] + b1;
+    }
+    __syncthreads();
+    for (int r = warp; r < 16; r += 4) {
+        const int64_t t = tok0 + r;
+        if (t >= T_tokens) break;
+        float logit[kSlots];
+#pragma unroll
+        for (int s = 0; s < kSlots; ++s) {
+            const int e = s * 32 + lane;
+            logit[s] = (s < kTilesPerWarp && e < E) ? s_logit[r][e] : -INFINITY;
+        }
+        softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs);
+    }
+}
+
+template <int kTilesPerWarp>
+void launch_route_mma(const monde_problem& p, const void* x, const void* Wg, const float* bg, int32_t* topk_idx,
+                      float* topk_w, float* probs, cudaStream_t s) {
+    route_mma_kernel<kTilesPerWarp><<<(p.T + 15) / 16, 128, 0, s>>>(
+        p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),
+        static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs);
+}
+
 // Histogram of assignments per expert (shared-memory atomics on integers: the sum does
 // not depend on order), then classification, compaction and exclusive scan by one warp.
 __global__ void __launch_bounds__(1024) histogram_classify_scan_kernel(
@@ -183,11 +266,12 @@ int launch_route(const monde_problem& p, const void* x, const void* Wg, const fl
                  int32_t* topk_idx, float* topk_w, float* probs, cudaStream_t s) {
     const int warps = 4;
     const int grid = (p.T + warps - 1) / warps;
-    if (p.dtype == MONDE_BF16)
-        route_warp_per_token_kernel<__nv_bfloat16><<<grid, warps * 32, 0, s>>>(
-            p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),
-            static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs);
-    else
+    if (p.dtype == MONDE_BF16) {
+        if (p.E <= 32) launch_route_mma<1>(p, x, Wg, bg, topk_idx, topk_w, probs, s);
+        else if (p.E <= 64) launch_route_mma<2>(p, x, Wg, bg, topk_idx, topk_w, probs, s);
+        else if (p.E <= 128) launch_route_mma<4>(p, x, Wg, bg, topk_idx, topk_w, probs, s);
+        else launch_route_mma<8>(p, x, Wg, bg, topk_idx, topk_w, probs, s);
+    } else
         route_warp_per_token_kernel<float><<<grid, warps * 32, 0, s>>>(
             p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const float*>(x),
             static_cast<const float*>(Wg), bg, topk_idx, topk_w, probs);
