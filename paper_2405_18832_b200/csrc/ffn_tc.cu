@@ -26,6 +26,7 @@
 // the second accumulator buffer.  Counts never travel to the host.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -33,11 +34,14 @@
 
 namespace monde {
 
+unsigned long long* g_trace = nullptr;
+int g_trace_slots = 0;
+
 namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;       // producer, MMA, 4 epilogue warps, publisher
 constexpr int kBlockK = 64;           // K elements per stage: one 128-byte swizzle row
 constexpr int kTileRows = 128;        // output features per unit = MMA M
 constexpr int kABytes = kTileRows * 128;
@@ -45,9 +49,10 @@ constexpr int kMaxStages = 8;
 constexpr int kHotTokTile = 256, kHotStages = 4;     // 4 x (16 KB + 32 KB)
 constexpr int kColdTokTile = 64, kColdStages = 8;    // 8 x (16 KB +  8 KB)
 constexpr int kTileBytes = 192 * 1024;
-constexpr int kNumBars = 2 * kMaxStages + 4;
+constexpr int kNumBars = 2 * kMaxStages + 6;
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
-constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kTableInts * 4;
+constexpr int kStageOutBytes = 2 * 16 * kTileRows * 2;
+constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kTableInts * 4 + kStageOutBytes + 16;
 constexpr int kTmemCols = 512;        // two accumulator buffers of 256 fp32 columns
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
 
@@ -67,8 +72,21 @@ struct FfnParams {
     const int32_t* n_hot_cold;
     int32_t* status;       // {status, site}
     int32_t* ticket;       // CTAs that have finished
-    int32_t* ready;        // per token tile: first-layer units finished (x4, one per epilogue warp)
+    int32_t* ready;        // per token tile: first-layer units finished
+    unsigned long long* trace;   // diagnostic timeline (null in normal use): [cta][unit slot][8]
+    int trace_slots;
 };
+
+// Diagnostic timeline: slot 0 unit id, 1-2 producer first/last issue, 3-4 MMA first full / commit,
+// 5-6 epilogue start / end (global timer, ns).
+__device__ __forceinline__ void trace_mark(const FfnParams& P, int it, int slot, unsigned long long v) {
+    if (P.trace != nullptr && it < P.trace_slots)
+        P.trace[(static_cast<size_t>(blockIdx.x) * P.trace_slots + it) * 8 + slot] = v;
+}
+__device__ __forceinline__ void trace_time(const FfnParams& P, int it, int slot) {
+    if (P.trace != nullptr && it < P.trace_slots)
+        P.trace[(static_cast<size_t>(blockIdx.x) * P.trace_slots + it) * 8 + slot] = global_timer_ns();
+}
 
 struct Unit {
     int e;        // expert id
@@ -126,6 +144,24 @@ __device__ __forceinline__ void report_timeout(int32_t* status, volatile int* ab
     if (atomicCAS(status, 0, MONDE_ERR_TIMEOUT) == 0) status[1] = site;
 }
 
+// erf by the rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7, far
+// below one bf16 rounding of the result); a dozen instructions instead of a library call.
+__device__ __forceinline__ float erf_as(float x) {
+    const float ax = fabsf(x);
+    const float t = __frcp_rn(fmaf(0.3275911f, ax, 1.0f));
+    float p = fmaf(1.061405429f, t, -1.453152027f);
+    p = fmaf(p, t, 1.421413741f);
+    p = fmaf(p, t, -0.284496736f);
+    p = fmaf(p, t, 0.254829592f);
+    const float r = 1.0f - p * t * __expf(-ax * ax);
+    return copysignf(r, x);
+}
+template <int kAct>
+__device__ __forceinline__ float activate(float v) {
+    if (kAct == MONDE_ACT_RELU) return fmaxf(v, 0.0f);
+    return 0.5f * v * (1.0f + erf_as(v * 0.70710678118654752440f));
+}
+
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -133,6 +169,7 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
+template <int kAct>
 __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
         const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_h, const FfnParams P) {
@@ -142,6 +179,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* tab = reinterpret_cast<int*>(tmem_slot + 16);
+    __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(                     // 2 x [16 tokens][128 features]
+        (reinterpret_cast<uintptr_t>(tab + kTableInts) + 15) & ~uintptr_t(15));
     UnitTable ut;
     ut.tt_prefix = tab;
     ut.e = tab + (kMaxExperts + 1);
@@ -180,6 +219,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bars[2 * kMaxStages + b]), 1);       // accumulator full: one commit
             mbar_init(smem_u32(&bars[2 * kMaxStages + 2 + b]), 4);   // accumulator drained: 4 epilogue warps
+            mbar_init(smem_u32(&bars[2 * kMaxStages + 4 + b]), 4);   // output rows stored: 4 epilogue warps
         }
         fence_barrier_init();
     }
@@ -221,7 +261,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     ut.seg[4] = ut.seg[3] + (tt_all - tt_hot) * ut.nt2;
     const int total_units = ut.seg[4];
     const uint32_t tiles_u32 = smem_u32(smem);
-    const int ready_target = 4 * ut.nt1;
+    const int ready_target = ut.nt1;
 
     if (warp == 0) {
         // ---- TMA producer ------------------------------------------------------------
@@ -235,8 +275,10 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             int stage = 0, cls = -1, stages = kHotStages, stage_bytes = kABytes + kHotTokTile * 128;
             uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
             bool ok = true;
-            for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
+            int pit = 0;
+            for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x, ++pit) {
                 const Unit un = ut.decode(u);
+                trace_mark(P, pit, 0, static_cast<unsigned long long>(u));
                 if (un.cold != cls) {
                     // geometry switch: every stage filled so far must have been consumed
                     for (int s = 0; ok && s < stages; ++s)
@@ -263,6 +305,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                         ok = false;
                         break;
                     }
+                    if (kb == 0) trace_time(P, pit, 1);
                     const uint32_t full = smem_u32(&bars[stage]);
                     const uint32_t a_dst = tiles_u32 + stage * stage_bytes;
                     mbar_arrive_expect_tx(full, kABytes + un.nt * 128);
@@ -288,6 +331,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     fill_bits ^= 1u << stage;
                     if (++stage == stages) stage = 0;
                 }
+                trace_time(P, pit, 2);
             }
         }
     } else if (warp == 1) {
@@ -321,6 +365,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                         break;
                     }
                     tc_fence_after_sync();
+                    if (kb == 0) trace_time(P, it, 3);
                     const uint32_t a_addr = tiles_u32 + stage * stage_bytes;
                     const uint64_t a_desc = smem_desc_sw128(a_addr);
                     const uint64_t b_desc = smem_desc_sw128(a_addr + kABytes);
@@ -332,9 +377,10 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     if (++stage == stages) stage = 0;
                 }
                 if (ok) umma_commit(smem_u32(&bars[2 * kMaxStages + b]));   // accumulator complete
+                trace_time(P, it, 4);
             }
         }
-    } else {
+    } else if (warp < 6) {
         // ---- epilogue: TMEM -> registers -> bias, activation -> global ----------------
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         int it = 0;
@@ -342,45 +388,99 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             const Unit un = ut.decode(u);
             const int b = it & 1;
             const uint32_t tphase = (it >> 1) & 1;
-            if (!mbar_wait(smem_u32(&bars[2 * kMaxStages + b]), tphase, abort_flag, kWaitLimitNs)) {
-                report_timeout(P.status, abort_flag, kSiteEpilogueTmemFull);
-                break;
-            }
+            const bool got = mbar_wait(smem_u32(&bars[2 * kMaxStages + b]), tphase, abort_flag, kWaitLimitNs);
+            if (!got) report_timeout(P.status, abort_flag, kSiteEpilogueTmemFull);
+            // the four epilogue warps share a named barrier below: leave together or not at all
+            uint32_t all_got;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.u32 q, %1, 0;\n\t"
+                "bar.red.and.pred p, 1, 128, q;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(all_got) : "r"(static_cast<uint32_t>(got)) : "memory");
+            if (!all_got) break;
             tc_fence_after_sync();
+            if (warp == 2 && lane == 0) trace_time(P, it, 5);
             const int N = un.layer ? P.d_model : P.d_ff;
-            const int act = un.layer ? -1 : P.act;
             const __nv_bfloat16* bias = un.layer ? P.b2 : P.b1;
             const int n = un.n0 + q * 32 + lane;
-            const bool n_ok = n < N;
-            const float bias_v = (bias != nullptr && n_ok) ? __bfloat162float(bias[static_cast<int64_t>(un.e) * N + n]) : 0.0f;
+            const float bias_v = (bias != nullptr && n < N) ? __bfloat162float(bias[static_cast<int64_t>(un.e) * N + n]) : 0.0f;
             const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 256;
-            __nv_bfloat16* dst = (un.layer ? P.y : P.h) + static_cast<int64_t>(un.row0) * N + n;
-            for (int c0 = 0; c0 < un.nt; c0 += 16) {
-                uint32_t v[16];
-                tmem_ld_16(t_addr + c0, v);
-                tmem_ld_wait();
-                if (n_ok) {
+            __nv_bfloat16* out = un.layer ? P.y : P.h;
+            const int et = tid - 64;                    // 0..127 within the epilogue warps (warps 2-5)
+            const int rd_row = et >> 4, rd_col = (et & 15) * 8;
+            const bool col_ok = un.n0 + rd_col < N;     // N is a multiple of 64: 8-wide groups are all in or all out
+            // 32 accumulator columns (tokens) per TMEM load, the next load in flight while this one
+            // is converted; each group of 16 tokens is transposed through shared memory so that
+            // global stores are 16-byte pieces of 256-byte contiguous row segments.  The code is
+            // kept small on purpose: an unrolled epilogue with an inlined library erf per element
+            // overflowed the instruction cache and ran 20x slower.
+            auto drain32 = [&](const uint32_t (&v)[32], int c32) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        if (c0 + j < un.rows) {
-                            float r = __uint_as_float(v[j]) + bias_v;
-                            if (act >= 0) r = apply_act(r, act);
-                            dst[static_cast<int64_t>(c0 + j) * N] = __float2bfloat16_rn(r);
+                for (int g = 0; g < 2; ++g) {
+                    const int c0 = c32 + g * 16;
+                    if (c0 < un.nt) {
+                        __nv_bfloat16* sb = stg + g * (16 * kTileRows);
+                        if (un.layer) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                sb[j * kTileRows + q * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[g * 16 + j]) + bias_v);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                sb[j * kTileRows + q * 32 + lane] =
+                                    __float2bfloat16_rn(activate<kAct>(__uint_as_float(v[g * 16 + j]) + bias_v));
+                        }
+                        asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            const int r = rd_row + half * 8;
+                            if (col_ok && c0 + r < un.rows) {
+                                const uint4 val = *reinterpret_cast<const uint4*>(sb + r * kTileRows + rd_col);
+                                *reinterpret_cast<uint4*>(out + static_cast<int64_t>(un.row0 + c0 + r) * N + un.n0 + rd_col) = val;
+                            }
                         }
                     }
                 }
+            };
+            uint32_t va[32], vb[32];
+            tmem_ld_32(t_addr, va);
+            for (int c32 = 0; c32 < un.nt; c32 += 64) {
+                tmem_ld_wait();
+                if (c32 + 32 < un.nt) tmem_ld_32(t_addr + c32 + 32, vb);
+                drain32(va, c32);
+                if (c32 + 32 < un.nt) {
+                    tmem_ld_wait();
+                    if (c32 + 64 < un.nt) tmem_ld_32(t_addr + c32 + 64, va);
+                    drain32(vb, c32 + 32);
+                }
             }
             tc_fence_before_sync();
-            if (un.layer == 0) {
-                // publish the hidden rows: stores visible device-wide (and to the async proxy
-                // that will read them through TMA) before the counter moves
-                __threadfence();
-                fence_proxy_async_all();
-            }
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(smem_u32(&bars[2 * kMaxStages + 2 + b]));
-                if (un.layer == 0) atomicAdd(P.ready + un.ready_idx, 1);
+                mbar_arrive(smem_u32(&bars[2 * kMaxStages + 2 + b]));   // accumulator buffer free
+                mbar_arrive(smem_u32(&bars[2 * kMaxStages + 4 + b]));   // rows stored (release, CTA scope)
+                if (warp == 2) trace_time(P, it, 6);
+            }
+        }
+    } else if (warp == 6) {
+        // ---- publisher: makes finished hidden rows visible device-wide -------------------
+        // The device-scope fence has to wait until the epilogue's stores have reached L2, which
+        // takes microseconds while TMA loads saturate the memory system; doing it here keeps
+        // that wait off the epilogue warps.  Order: epilogue stores -> mbarrier (release/acquire
+        // at CTA scope) -> this thread's device-scope fence (cumulative) -> counter increment.
+        if (lane == 0) {
+            int it = 0;
+            for (int u = blockIdx.x; u < total_units; u += gridDim.x, ++it) {
+                const Unit un = ut.decode(u);
+                const int b = it & 1;
+                if (!mbar_wait(smem_u32(&bars[2 * kMaxStages + 4 + b]), (it >> 1) & 1, abort_flag, kWaitLimitNs))
+                    break;   // the role that stalled has already reported
+                if (un.layer == 0) {
+                    __threadfence();
+                    fence_proxy_async_all();
+                    atomicAdd(P.ready + un.ready_idx, 1);
+                }
             }
         }
     }
@@ -457,7 +557,11 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(expert_ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        attr_err = cudaFuncSetAttribute(expert_ffn_kernel<MONDE_ACT_RELU>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(expert_ffn_kernel<MONDE_ACT_GELU_ERF>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     });
     if (attr_err != cudaSuccess) return MONDE_ERR_CUDA;
     char* base = static_cast<char*>(ws);
@@ -478,13 +582,25 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.status = reinterpret_cast<int32_t*>(base + WsLayout::kStatus);
     P.ticket = reinterpret_cast<int32_t*>(base + WsLayout::kCounters);
     P.ready = reinterpret_cast<int32_t*>(base + WsLayout::kTiles);
+    P.trace = g_trace;
+    P.trace_slots = g_trace_slots;
     CUtensorMap map_w1, map_w2, map_x, map_h;
     if (!make_map(&map_w1, W1, static_cast<uint64_t>(p.E) * p.d_ff, p.d_model, kTileRows)) return MONDE_ERR_CUDA;
     if (!make_map(&map_w2, W2, static_cast<uint64_t>(p.E) * p.d_model, p.d_ff, kTileRows)) return MONDE_ERR_CUDA;
     if (!make_map(&map_x, x_perm, A, p.d_model, 16)) return MONDE_ERR_CUDA;
     if (!make_map(&map_h, P.h, A, p.d_ff, 16)) return MONDE_ERR_CUDA;
-    expert_ffn_kernel<<<sm_count(), kThreads, kSmemBytes, s>>>(map_w1, map_w2, map_x, map_h, P);
+    if (p.act == MONDE_ACT_RELU)
+        expert_ffn_kernel<MONDE_ACT_RELU><<<sm_count(), kThreads, kSmemBytes, s>>>(map_w1, map_w2, map_x, map_h, P);
+    else
+        expert_ffn_kernel<MONDE_ACT_GELU_ERF><<<sm_count(), kThreads, kSmemBytes, s>>>(map_w1, map_w2, map_x, map_h, P);
     return launched();
 }
 
 }  // namespace monde
+
+// Diagnostic hook (not part of the public header): device buffer of 148 * slots * 8 uint64
+// that the FFN kernel fills with a per-unit timeline; pass null to switch it off.
+extern "C" void monde_internal_set_trace(void* device_buf, int slots) {
+    monde::g_trace = static_cast<unsigned long long*>(device_buf);
+    monde::g_trace_slots = slots;
+}
