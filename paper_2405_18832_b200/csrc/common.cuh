@@ -23,6 +23,11 @@ struct WsLayout {
     static constexpr size_t kTilesBytes = 112 * 1024;
     static constexpr size_t kHidden = 128 * 1024;  // h [A, d_ff] in the problem dtype
     size_t hidden_bytes;
+    int n_split;            // K-splits of a cold second-layer unit
+    size_t part_done_off;   // int32 per cold second-layer tile (zero between calls)
+    size_t part_done_bytes;
+    size_t partials_off;    // fp32 partial tiles of the K-split cold second-layer units
+    size_t partials_bytes;
     size_t total;
 };
 // The header (first kHidden bytes) holds everything that must be zero between calls: the
@@ -33,11 +38,33 @@ static_assert(4 * (kMaxAssignments / 64 + 2 * 256 + 64) <= 112 * 1024, "token-ti
 
 inline size_t elem_bytes(int dtype) { return dtype == MONDE_BF16 ? 2 : 4; }
 
+// Token-tile width of the cold class: a cold expert has at most hot_threshold-1 rows.
+inline int cold_token_tile(const monde_problem& p) {
+    const long long t = (static_cast<long long>(p.hot_threshold) - 1 + 15) / 16 * 16;
+    return static_cast<int>(t < 16 ? 16 : (t > 64 ? 64 : t));
+}
+
 inline WsLayout ws_layout(const monde_problem& p) {
     WsLayout l;
     size_t A = static_cast<size_t>(p.T) * p.top_k;
     l.hidden_bytes = (A * p.d_ff * elem_bytes(p.dtype) + 1023) / 1024 * 1024;
-    l.total = WsLayout::kHidden + l.hidden_bytes + 1024;
+    // Cold second-layer units are split along K when d_ff is a multiple of d_model's size and
+    // the partial tiles fit a bounded scratch (otherwise no split).
+    const size_t ct = cold_token_tile(p);
+    const size_t nt2 = (static_cast<size_t>(p.d_model) + 127) / 128;
+    const size_t cold_tiles = (A / ct + p.E) * nt2;          // upper bound on cold second-layer tiles
+    int split = p.d_ff / p.d_model;
+    split = split < 1 ? 1 : (split > 4 ? 4 : split);
+    const int kb2 = p.d_ff / 64;                              // every sub-unit must own at least one K block
+    while (split > 1 && (split - 1) * ((kb2 + split - 1) / split) >= kb2) --split;
+    size_t part = cold_tiles * (split - 1) * ct * 128 * 4;
+    if (part > (size_t(1) << 30)) { split = 1; part = 0; }
+    l.n_split = split;
+    l.part_done_off = WsLayout::kHidden + l.hidden_bytes;
+    l.part_done_bytes = split > 1 ? (cold_tiles * 4 + 1023) / 1024 * 1024 : 0;
+    l.partials_off = l.part_done_off + l.part_done_bytes;
+    l.partials_bytes = part;
+    l.total = l.partials_off + l.partials_bytes + 1024;
     return l;
 }
 

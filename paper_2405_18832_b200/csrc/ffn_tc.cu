@@ -13,20 +13,27 @@
 // so an expert with m tokens costs one pass over its weights with N = m rounded up to 16.
 // The class chosen by the router selects the tiling of a work unit:
 //   hot : token tile <= 256 (a full-rate 128 x 256 MMA), 4-stage ring of 48 KB stages;
-//   cold: token tile <= 64, 8-stage ring of 24 KB stages -> a deep queue of weight bytes in
-//         flight per SM; the tensor core idles most of the time and HBM sets the pace.
-// Work units (expert, 128-feature tile, token tile) are ordered hot-first-layer,
-// hot-second-layer, cold-first-layer, cold-second-layer and dealt round-robin to one
-// persistent CTA per SM.  A second-layer unit needs the hidden rows of its token tile,
-// which are produced by first-layer units earlier in the same order: per-token-tile
-// counters in the workspace carry that dependency, and the TMA producer streams the
-// unit's weights while it waits, so weight traffic never stalls at the layer boundary.
+//   cold: token tile = threshold-1 rounded up to 16 (at most 64), 8 to 10 stages of 18-24 KB
+//         -> a deep queue of weight bytes in flight per SM; the tensor core idles most of
+//         the time and HBM sets the pace.
+// Work units (expert, 128-feature tile, token tile) form one ordered list: hot first
+// layer, hot second layer, cold first layer, cold second layer.  One persistent CTA per SM
+// takes the next unit from a device-wide counter.  A second-layer unit needs the hidden
+// rows of its token tile, which are produced by first-layer units earlier in the list:
+// per-token-tile counters in the workspace carry that dependency (a unit only ever waits
+// for units taken before it, so the wait cannot deadlock), and the TMA producer streams
+// the unit's weights while it waits, so weight traffic never stalls at the layer boundary.
+// Cold second-layer units are long (K = d_ff) and few; they are split along K into up to
+// four sub-units so that the end of the run is not a handful of CTAs each streaming a
+// megabyte alone.  Sub-units 0..S-2 store fp32 partial tiles in the workspace; the last
+// sub-unit (again later in the list than the ones it waits for) adds them in a fixed
+// order, so results stay bit-reproducible.
 // Warp roles: warp 0 issues TMA, warp 1 issues MMAs and owns the TMEM allocation, warps
 // 2-5 drain the accumulator (bias + activation fused) while the next unit's MMAs run into
 // the second accumulator buffer.  Counts never travel to the host.
 #include <cuda.h>
 
-#include <cstdlib>
+#include <algorithm>
 #include <mutex>
 
 #include "common.cuh"
@@ -45,11 +52,11 @@ constexpr int kThreads = 224;       // producer, MMA, 4 epilogue warps, publishe
 constexpr int kBlockK = 64;           // K elements per stage: one 128-byte swizzle row
 constexpr int kTileRows = 128;        // output features per unit = MMA M
 constexpr int kABytes = kTileRows * 128;
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 10;
+constexpr int kQueue = 4;            // unit ids in flight between the producer and the other roles
 constexpr int kHotTokTile = 256, kHotStages = 4;     // 4 x (16 KB + 32 KB)
-constexpr int kColdTokTile = 64, kColdStages = 8;    // 8 x (16 KB +  8 KB)
 constexpr int kTileBytes = 192 * 1024;
-constexpr int kNumBars = 2 * kMaxStages + 6;
+constexpr int kNumBars = 2 * kMaxStages + 6 + 2 * kQueue;
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
 constexpr int kStageOutBytes = 2 * 16 * kTileRows * 2;
 constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kTableInts * 4 + kStageOutBytes + 16;
@@ -57,10 +64,12 @@ constexpr int kTmemCols = 512;        // two accumulator buffers of 256 fp32 col
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
 
 enum WaitSite { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4,
-                kSiteHiddenReady = 5, kSiteDrain = 6 };
+                kSiteHiddenReady = 5, kSiteDrain = 6, kSiteQueue = 7, kSitePartials = 8 };
 
 struct FfnParams {
     int d_model, d_ff, act;
+    int cold_tile, cold_stages;   // stage geometry of the cold class
+    int n_split;                  // K-splits of a cold second-layer unit (1 = none)
     const __nv_bfloat16* b1;
     const __nv_bfloat16* b2;
     __nv_bfloat16* h;
@@ -72,6 +81,9 @@ struct FfnParams {
     const int32_t* n_hot_cold;
     int32_t* status;       // {status, site}
     int32_t* ticket;       // CTAs that have finished
+    int32_t* next_unit;    // device-wide unit counter
+    int32_t* part_done;    // per cold second-layer tile: partial tiles finished
+    float* partials;       // [tile][split][cold_tile tokens][128 features] fp32
     int32_t* ready;        // per token tile: first-layer units finished
     unsigned long long* trace;   // diagnostic timeline (null in normal use): [cta][unit slot][8]
     int trace_slots;
@@ -97,6 +109,10 @@ struct Unit {
     int layer;    // 0: h = act(x W1^T + b1), 1: y = h W2^T + b2
     int cold;     // class: selects the stage geometry
     int ready_idx;  // token-tile index into the dependency counters
+    int kb0, kb1;   // K blocks [kb0, kb1) of the reduction handled by this unit
+    int split;      // sub-unit index along K, n_split - 1 = the one that finishes the tile
+    int n_split;    // sub-units of this tile (1 unless cold second layer)
+    int tile_idx;   // cold second-layer tile index (partials / part_done)
 };
 
 // Per-CTA copy of the unit list in shared memory.  Entries 0..n_hot-1 are the hot experts,
@@ -109,18 +125,27 @@ struct UnitTable {
     int* tt;          // token tiles of this expert
     int* per;         // tokens per tile (multiple of 16)
     int n_hot, n_all, nt1, nt2;      // 128-feature tiles of layer 1 (d_ff) and layer 2 (d_model)
-    int seg[5];                      // unit index where each (class, layer) segment starts
+    int kblocks1, kblocks2;          // 64-wide K blocks of layer 1 (d_model) and layer 2 (d_ff)
+    int n_split, kb_per_split;
+    int seg1, seg2, seg3, total_units;   // list = [hot L1 | hot L2 | cold L1 | cold L2 (split)]
 
     __device__ __forceinline__ Unit decode(int u) const {
-        int sgm = 0;
-        while (u >= seg[sgm + 1]) ++sgm;
         Unit r;
-        r.cold = sgm >> 1;
-        r.layer = sgm & 1;
+        int v;
+        if (u < seg1) { r.cold = 0; r.layer = 0; v = u; }
+        else if (u < seg2) { r.cold = 0; r.layer = 1; v = u - seg1; }
+        else if (u < seg3) { r.cold = 1; r.layer = 0; v = u - seg2; }
+        else { r.cold = 1; r.layer = 1; v = u - seg3; }
+        r.split = 0;
+        r.n_split = 1;
+        if (r.cold && r.layer) {
+            r.n_split = n_split;
+            r.split = v % n_split;
+            v /= n_split;
+        }
         const int ntl = r.layer ? nt2 : nt1;
         const int lo_entry = r.cold ? n_hot : 0;
         const int tt_base = tt_prefix[lo_entry];
-        const int v = u - seg[sgm];
         int lo = lo_entry, hi = (r.cold ? n_all : n_hot) - 1;      // largest entry with block start <= v
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
@@ -128,13 +153,18 @@ struct UnitTable {
         }
         const int local = v - (tt_prefix[lo] - tt_base) * ntl;
         const int tok = local % tt[lo];
+        const int ntile = local / tt[lo];
         r.e = e[lo];
-        r.n0 = (local / tt[lo]) * kTileRows;
+        r.n0 = ntile * kTileRows;
         const int r_in_e = tok * per[lo];
         r.rows = min(per[lo], m[lo] - r_in_e);
         r.nt = (r.rows + 15) & ~15;
         r.row0 = off[lo] + r_in_e;
         r.ready_idx = tt_prefix[lo] + tok;
+        r.tile_idx = (tt_prefix[lo] - tt_base + tok) * nt2 + ntile;
+        const int kb_all = r.layer ? kblocks2 : kblocks1;
+        r.kb0 = r.n_split > 1 ? r.split * kb_per_split : 0;
+        r.kb1 = r.n_split > 1 ? min(kb_all, r.kb0 + kb_per_split) : kb_all;
         return r;
     }
 };
@@ -178,6 +208,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTileBytes);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* unit_queue = reinterpret_cast<volatile int*>(tmem_slot + 4);      // [kQueue]
     int* tab = reinterpret_cast<int*>(tmem_slot + 16);
     __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(                     // 2 x [16 tokens][128 features]
         (reinterpret_cast<uintptr_t>(tab + kTableInts) + 15) & ~uintptr_t(15));
@@ -189,6 +220,16 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     ut.tt = ut.m + (kMaxExperts + 1);
     ut.per = ut.tt + (kMaxExperts + 1);
 
+    // barrier addresses
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+    auto acc_full = [&](int b) { return bar0 + 8u * (2 * kMaxStages + b); };
+    auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 2 + b); };
+    auto rows_stored = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 4 + b); };
+    auto q_full = [&](int s) { return bar0 + 8u * (2 * kMaxStages + 6 + s); };
+    auto q_empty = [&](int s) { return bar0 + 8u * (2 * kMaxStages + 6 + kQueue + s); };
+
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     ut.n_hot = min(P.n_hot_cold[0], kMaxExperts);
     ut.n_all = min(ut.n_hot + P.n_hot_cold[1], kMaxExperts);
@@ -199,7 +240,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     for (int i = tid; i < ut.n_all; i += kThreads) {
         const bool cold = i >= ut.n_hot;
         const int e = cold ? P.cold_ids[i - ut.n_hot] : P.hot_ids[i];
-        const int tile = cold ? kColdTokTile : kHotTokTile;
+        const int tile = cold ? P.cold_tile : kHotTokTile;
         const int m = P.counts[e];
         const int tt = max(1, (m + tile - 1) / tile);
         ut.e[i] = e;
@@ -213,13 +254,17 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         ut.tt_prefix[0] = 0;
         *abort_flag = 0;
         for (int s = 0; s < kMaxStages; ++s) {
-            mbar_init(smem_u32(&bars[s]), 1);               // full: producer's expect_tx arrival
-            mbar_init(smem_u32(&bars[kMaxStages + s]), 1);  // empty: one tcgen05.commit
+            mbar_init(full_bar(s), 1);    // producer's expect_tx arrival
+            mbar_init(empty_bar(s), 1);   // one tcgen05.commit
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&bars[2 * kMaxStages + b]), 1);       // accumulator full: one commit
-            mbar_init(smem_u32(&bars[2 * kMaxStages + 2 + b]), 4);   // accumulator drained: 4 epilogue warps
-            mbar_init(smem_u32(&bars[2 * kMaxStages + 4 + b]), 4);   // output rows stored: 4 epilogue warps
+            mbar_init(acc_full(b), 1);      // one commit
+            mbar_init(acc_empty(b), 4);     // 4 epilogue warps
+            mbar_init(rows_stored(b), 4);   // 4 epilogue warps
+        }
+        for (int s = 0; s < kQueue; ++s) {
+            mbar_init(q_full(s), 1);        // producer
+            mbar_init(q_empty(s), 6);       // MMA issuer, 4 epilogue warps, publisher
         }
         fence_barrier_init();
     }
@@ -253,18 +298,35 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const int tt_hot = ut.tt_prefix[ut.n_hot], tt_all = ut.tt_prefix[ut.n_all];
-    ut.seg[0] = 0;
-    ut.seg[1] = tt_hot * ut.nt1;
-    ut.seg[2] = ut.seg[1] + tt_hot * ut.nt2;
-    ut.seg[3] = ut.seg[2] + (tt_all - tt_hot) * ut.nt1;
-    ut.seg[4] = ut.seg[3] + (tt_all - tt_hot) * ut.nt2;
-    const int total_units = ut.seg[4];
+    const int tt_all = ut.tt_prefix[ut.n_all];
+    const int tt_hot = ut.tt_prefix[ut.n_hot];
+    ut.kblocks1 = P.d_model / kBlockK;
+    ut.kblocks2 = P.d_ff / kBlockK;
+    ut.n_split = P.n_split;
+    ut.kb_per_split = (ut.kblocks2 + P.n_split - 1) / P.n_split;
+    ut.seg1 = tt_hot * ut.nt1;
+    ut.seg2 = ut.seg1 + tt_hot * ut.nt2;
+    ut.seg3 = ut.seg2 + (tt_all - tt_hot) * ut.nt1;
+    ut.total_units = ut.seg3 + (tt_all - tt_hot) * ut.nt2 * P.n_split;
     const uint32_t tiles_u32 = smem_u32(smem);
     const int ready_target = ut.nt1;
+    const int cold_stage_bytes = kABytes + P.cold_tile * 128;
+    const int hot_stage_bytes = kABytes + kHotTokTile * 128;
+
+    // Every role but the producer takes its next unit id from the shared-memory queue.
+    // Returns -1 at the end of the list or when a wait gave up.
+    // `whole_warp`: all 32 lanes call (epilogue warps); otherwise a single lane calls.
+    auto pop_unit = [&](int it, bool whole_warp) -> int {
+        const int slot = it % kQueue;
+        if (!mbar_wait(q_full(slot), (it / kQueue) & 1, abort_flag, kWaitLimitNs)) return -1;
+        const int u = unit_queue[slot];
+        if (whole_warp) __syncwarp();
+        if (lane == 0) mbar_arrive(q_empty(slot));
+        return u;
+    };
 
     if (warp == 0) {
-        // ---- TMA producer ------------------------------------------------------------
+        // ---- scheduler + TMA producer ------------------------------------------------------
         if (lane == 0) {
             prefetch_tensormap(&map_w1);
             prefetch_tensormap(&map_w2);
@@ -272,45 +334,52 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             prefetch_tensormap(&map_h);
             const uint64_t pol_w = policy_evict_first();   // weights are read once
             const uint64_t pol_x = policy_evict_last();    // token tiles are re-read by every feature tile
-            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = kABytes + kHotTokTile * 128;
+            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes;
             uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
             bool ok = true;
-            int pit = 0;
-            for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x, ++pit) {
+            int u_next = atomicAdd(P.next_unit, 1);     // one id ahead: hides the atomic's round trip
+            for (int it = 0; ok; ++it) {
+                const int slot = it % kQueue;
+                if (!mbar_wait(q_empty(slot), ((it / kQueue) & 1) ^ 1, abort_flag, kWaitLimitNs)) {
+                    report_timeout(P.status, abort_flag, kSiteQueue);
+                    break;
+                }
+                int u = u_next;
+                if (u >= ut.total_units) u = -1;
+                else u_next = atomicAdd(P.next_unit, 1);
+                unit_queue[slot] = u;
+                mbar_arrive(q_full(slot));          // release: the id is visible to whoever acquires
+                if (u < 0) break;
                 const Unit un = ut.decode(u);
-                trace_mark(P, pit, 0, static_cast<unsigned long long>(u));
+                trace_mark(P, it, 0, static_cast<unsigned long long>(u));
                 if (un.cold != cls) {
                     // geometry switch: every stage filled so far must have been consumed
                     for (int s = 0; ok && s < stages; ++s)
-                        if (!mbar_wait(smem_u32(&bars[kMaxStages + s]), ((fill_bits >> s) & 1u) ^ 1u, abort_flag,
-                                       kWaitLimitNs)) {
+                        if (!mbar_wait(empty_bar(s), ((fill_bits >> s) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                             report_timeout(P.status, abort_flag, kSiteDrain);
                             ok = false;
                         }
                     if (!ok) break;
                     cls = un.cold;
-                    stages = cls ? kColdStages : kHotStages;
-                    stage_bytes = kABytes + (cls ? kColdTokTile : kHotTokTile) * 128;
+                    stages = cls ? P.cold_stages : kHotStages;
+                    stage_bytes = cls ? cold_stage_bytes : hot_stage_bytes;
                     stage = 0;
                 }
                 const CUtensorMap* mw = un.layer ? &map_w2 : &map_w1;
                 const CUtensorMap* mi = un.layer ? &map_h : &map_x;
-                const int K = un.layer ? P.d_ff : P.d_model;
                 const int N = un.layer ? P.d_model : P.d_ff;
-                const int k_blocks = K / kBlockK;
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!mbar_wait(smem_u32(&bars[kMaxStages + stage]), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag,
-                                   kWaitLimitNs)) {
+                for (int kb = un.kb0; kb < un.kb1; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteProducerEmpty);
                         ok = false;
                         break;
                     }
-                    if (kb == 0) trace_time(P, pit, 1);
-                    const uint32_t full = smem_u32(&bars[stage]);
+                    if (kb == un.kb0) trace_time(P, it, 1);
+                    const uint32_t full = full_bar(stage);
                     const uint32_t a_dst = tiles_u32 + stage * stage_bytes;
                     mbar_arrive_expect_tx(full, kABytes + un.nt * 128);
                     tma_load_2d(a_dst, mw, full, kb * kBlockK, un.e * N + un.n0, pol_w);
-                    if (kb == 0 && un.layer == 1) {
+                    if (kb == un.kb0 && un.layer == 1) {
                         // the hidden rows of this token tile must be complete; weights already stream
                         const int32_t* flag = P.ready + un.ready_idx;
                         if (ld_acquire(flag) < ready_target) {
@@ -331,65 +400,70 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     fill_bits ^= 1u << stage;
                     if (++stage == stages) stage = 0;
                 }
-                trace_time(P, pit, 2);
+                trace_time(P, it, 2);
             }
         }
     } else if (warp == 1) {
         // ---- MMA issuer --------------------------------------------------------------
         if (lane == 0) {
-            int stage = 0, it = 0, cls = -1, stages = kHotStages, stage_bytes = kABytes + kHotTokTile * 128;
+            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes;
             uint32_t use_bits = 0;      // bit s: parity of the number of uses of stage s
             bool ok = true;
-            for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x, ++it) {
+            for (int it = 0; ok; ++it) {
+                const int u = pop_unit(it, false);
+                if (u < 0) break;
                 const Unit un = ut.decode(u);
                 if (un.cold != cls) {
                     cls = un.cold;
-                    stages = cls ? kColdStages : kHotStages;
-                    stage_bytes = kABytes + (cls ? kColdTokTile : kHotTokTile) * 128;
+                    stages = cls ? P.cold_stages : kHotStages;
+                    stage_bytes = cls ? cold_stage_bytes : hot_stage_bytes;
                     stage = 0;
                 }
                 const int b = it & 1;
                 const uint32_t tphase = (it >> 1) & 1;
-                if (!mbar_wait(smem_u32(&bars[2 * kMaxStages + 2 + b]), tphase ^ 1u, abort_flag, kWaitLimitNs)) {
+                if (!mbar_wait(acc_empty(b), tphase ^ 1u, abort_flag, kWaitLimitNs)) {
                     report_timeout(P.status, abort_flag, kSiteMmaTmemEmpty);
                     break;
                 }
                 tc_fence_after_sync();
                 const uint32_t idesc = idesc_bf16_m128(un.nt);
                 const uint32_t d_tmem = tmem_base + b * 256;
-                const int k_blocks = (un.layer ? P.d_ff : P.d_model) / kBlockK;
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!mbar_wait(smem_u32(&bars[stage]), (use_bits >> stage) & 1u, abort_flag, kWaitLimitNs)) {
+                for (int kb = un.kb0; kb < un.kb1; ++kb) {
+                    if (!mbar_wait(full_bar(stage), (use_bits >> stage) & 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteMmaFull);
                         ok = false;
                         break;
                     }
                     tc_fence_after_sync();
-                    if (kb == 0) trace_time(P, it, 3);
+                    if (kb == un.kb0) trace_time(P, it, 3);
                     const uint32_t a_addr = tiles_u32 + stage * stage_bytes;
                     const uint64_t a_desc = smem_desc_sw128(a_addr);
                     const uint64_t b_desc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
                     for (int k4 = 0; k4 < kBlockK / 16; ++k4)
-                        umma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kb | k4) != 0);
-                    umma_commit(smem_u32(&bars[kMaxStages + stage]));   // stage reusable once these MMAs finish
+                        umma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kb != un.kb0) | (k4 != 0));
+                    umma_commit(empty_bar(stage));   // stage reusable once these MMAs finish
                     use_bits ^= 1u << stage;
                     if (++stage == stages) stage = 0;
                 }
-                if (ok) umma_commit(smem_u32(&bars[2 * kMaxStages + b]));   // accumulator complete
+                if (ok) umma_commit(acc_full(b));   // accumulator complete
                 trace_time(P, it, 4);
             }
         }
     } else if (warp < 6) {
-        // ---- epilogue: TMEM -> registers -> bias, activation -> global ----------------
+        // ---- epilogue: TMEM -> registers -> bias, activation -> shared -> global -------------
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
-        int it = 0;
-        for (int u = blockIdx.x; u < total_units; u += gridDim.x, ++it) {
-            const Unit un = ut.decode(u);
+        for (int it = 0;; ++it) {
+            const int u = pop_unit(it, true);
             const int b = it & 1;
             const uint32_t tphase = (it >> 1) & 1;
-            const bool got = mbar_wait(smem_u32(&bars[2 * kMaxStages + b]), tphase, abort_flag, kWaitLimitNs);
-            if (!got) report_timeout(P.status, abort_flag, kSiteEpilogueTmemFull);
+            bool got = u >= 0;
+            Unit un;
+            if (got) {
+                un = ut.decode(u);
+                got = mbar_wait(acc_full(b), tphase, abort_flag, kWaitLimitNs);
+                if (!got) report_timeout(P.status, abort_flag, kSiteEpilogueTmemFull);
+            }
             // the four epilogue warps share a named barrier below: leave together or not at all
             uint32_t all_got;
             asm volatile(
@@ -410,56 +484,93 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             const int et = tid - 64;                    // 0..127 within the epilogue warps (warps 2-5)
             const int rd_row = et >> 4, rd_col = (et & 15) * 8;
             const bool col_ok = un.n0 + rd_col < N;     // N is a multiple of 64: 8-wide groups are all in or all out
-            // 32 accumulator columns (tokens) per TMEM load, the next load in flight while this one
-            // is converted; each group of 16 tokens is transposed through shared memory so that
-            // global stores are 16-byte pieces of 256-byte contiguous row segments.  The code is
-            // kept small on purpose: an unrolled epilogue with an inlined library erf per element
-            // overflowed the instruction cache and ran 20x slower.
-            auto drain32 = [&](const uint32_t (&v)[32], int c32) {
-#pragma unroll
-                for (int g = 0; g < 2; ++g) {
-                    const int c0 = c32 + g * 16;
-                    if (c0 < un.nt) {
-                        __nv_bfloat16* sb = stg + g * (16 * kTileRows);
-                        if (un.layer) {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                sb[j * kTileRows + q * 32 + lane] = __float2bfloat16_rn(__uint_as_float(v[g * 16 + j]) + bias_v);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                sb[j * kTileRows + q * 32 + lane] =
-                                    __float2bfloat16_rn(activate<kAct>(__uint_as_float(v[g * 16 + j]) + bias_v));
-                        }
-                        asm volatile("bar.sync 1, 128;" ::: "memory");
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            const int r = rd_row + half * 8;
-                            if (col_ok && c0 + r < un.rows) {
-                                const uint4 val = *reinterpret_cast<const uint4*>(sb + r * kTileRows + rd_col);
-                                *reinterpret_cast<uint4*>(out + static_cast<int64_t>(un.row0 + c0 + r) * N + un.n0 + rd_col) = val;
-                            }
+            // Each group of 16 tokens is transposed through shared memory so that global stores are
+            // 16-byte pieces of 256-byte contiguous row segments.  The code is kept small on purpose:
+            // a widely unrolled epilogue with an inlined library erf per element overflowed the
+            // instruction cache and ran 20x slower.
+            // K-split tiles: fp32 partials live as [split][token][feature] so that a warp touches
+            // 128 contiguous bytes per token.
+            float* part = P.partials + static_cast<size_t>(un.tile_idx) * (un.n_split - 1) * (P.cold_tile * kTileRows) +
+                          q * 32 + lane;
+            const bool is_partial = un.split + 1 < un.n_split;
+            if (un.n_split > 1 && !is_partial) {
+                // finishing sub-unit: the partial tiles were taken from the list before this one
+                if (lane == 0) {
+                    const int32_t* flag = P.part_done + un.tile_idx;
+                    const uint64_t t0 = global_timer_ns();
+                    while (ld_acquire(flag) < un.n_split - 1) {
+                        if (*abort_flag != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
+                            report_timeout(P.status, abort_flag, kSitePartials);
+                            break;   // the sums below are wrong but every access stays in bounds
                         }
                     }
                 }
+                __syncwarp();
+            }
+            // One group = 16 tokens.  mode: 0 first layer (activation), 1 second layer, 2 second
+            // layer finishing a K-split tile (adds the partial tiles), 3 partial tile (fp32 store).
+            const int mode = un.layer == 0 ? 0 : (un.n_split == 1 ? 1 : (is_partial ? 3 : 2));
+            auto drain16 = [&](const uint32_t (&v)[16], int c0) {
+                if (mode == 3) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        part[(un.split * P.cold_tile + c0 + j) * kTileRows] = __uint_as_float(v[j]);
+                    return;
+                }
+                __nv_bfloat16* sb = stg + ((c0 >> 4) & 1) * (16 * kTileRows) + q * 32 + lane;
+                if (mode == 0) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        sb[j * kTileRows] = __float2bfloat16_rn(activate<kAct>(__uint_as_float(v[j]) + bias_v));
+                } else if (mode == 1) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        sb[j * kTileRows] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias_v);
+                } else {
+                    float acc[16];                                   // fixed order: split 0, 1, .., own
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
+#pragma unroll 1
+                    for (int sp = 0; sp + 1 < un.n_split; ++sp) {
+                        const float* ps = part + (sp * P.cold_tile + c0) * kTileRows;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) acc[j] += __ldcg(ps + j * kTileRows);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        sb[j * kTileRows] = __float2bfloat16_rn(acc[j] + __uint_as_float(v[j]) + bias_v);
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const __nv_bfloat16* rb = stg + ((c0 >> 4) & 1) * (16 * kTileRows);
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int r = rd_row + half * 8;
+                    if (col_ok && c0 + r < un.rows) {
+                        const uint4 val = *reinterpret_cast<const uint4*>(rb + r * kTileRows + rd_col);
+                        *reinterpret_cast<uint4*>(out + static_cast<int64_t>(un.row0 + c0 + r) * N + un.n0 + rd_col) = val;
+                    }
+                }
             };
-            uint32_t va[32], vb[32];
-            tmem_ld_32(t_addr, va);
-            for (int c32 = 0; c32 < un.nt; c32 += 64) {
+            // Two 16-column loads in flight, ping-pong; the loop is kept rolled so that the whole
+            // epilogue stays a few KB of code.
+            uint32_t va[16], vb[16];
+            tmem_ld_16(t_addr, va);
+#pragma unroll 1
+            for (int c0 = 0; c0 < un.nt; c0 += 32) {
                 tmem_ld_wait();
-                if (c32 + 32 < un.nt) tmem_ld_32(t_addr + c32 + 32, vb);
-                drain32(va, c32);
-                if (c32 + 32 < un.nt) {
+                if (c0 + 16 < un.nt) tmem_ld_16(t_addr + c0 + 16, vb);
+                drain16(va, c0);
+                if (c0 + 16 < un.nt) {
                     tmem_ld_wait();
-                    if (c32 + 64 < un.nt) tmem_ld_32(t_addr + c32 + 64, va);
-                    drain32(vb, c32 + 32);
+                    if (c0 + 32 < un.nt) tmem_ld_16(t_addr + c0 + 32, va);
+                    drain16(vb, c0 + 16);
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(smem_u32(&bars[2 * kMaxStages + 2 + b]));   // accumulator buffer free
-                mbar_arrive(smem_u32(&bars[2 * kMaxStages + 4 + b]));   // rows stored (release, CTA scope)
+                mbar_arrive(acc_empty(b));     // accumulator buffer free
+                mbar_arrive(rows_stored(b));   // rows stored (release, CTA scope)
                 if (warp == 2) trace_time(P, it, 6);
             }
         }
@@ -470,16 +581,20 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         // that wait off the epilogue warps.  Order: epilogue stores -> mbarrier (release/acquire
         // at CTA scope) -> this thread's device-scope fence (cumulative) -> counter increment.
         if (lane == 0) {
-            int it = 0;
-            for (int u = blockIdx.x; u < total_units; u += gridDim.x, ++it) {
+            for (int it = 0;; ++it) {
+                const int u = pop_unit(it, false);
+                if (u < 0) break;
                 const Unit un = ut.decode(u);
                 const int b = it & 1;
-                if (!mbar_wait(smem_u32(&bars[2 * kMaxStages + 4 + b]), (it >> 1) & 1, abort_flag, kWaitLimitNs))
+                if (!mbar_wait(rows_stored(b), (it >> 1) & 1, abort_flag, kWaitLimitNs))
                     break;   // the role that stalled has already reported
                 if (un.layer == 0) {
                     __threadfence();
                     fence_proxy_async_all();
                     atomicAdd(P.ready + un.ready_idx, 1);
+                } else if (un.split + 1 < un.n_split) {
+                    __threadfence();
+                    atomicAdd(P.part_done + un.tile_idx, 1);
                 }
             }
         }
@@ -492,7 +607,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }
-    // The last CTA to finish leaves the dependency counters at zero for the next call.
+    // The last CTA to finish leaves the counters at zero for the next call.
     if (warp == 2) {
         int last = 0;
         if (lane == 0) {
@@ -502,7 +617,12 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
             for (int i = lane; i < tt_all; i += 32) P.ready[i] = 0;
-            if (lane == 0) *P.ticket = 0;
+            if (P.n_split > 1)
+                for (int i = lane; i < (tt_all - tt_hot) * ut.nt2; i += 32) P.part_done[i] = 0;
+            if (lane == 0) {
+                *P.next_unit = 0;
+                *P.ticket = 0;
+            }
         }
     }
 }
@@ -581,6 +701,13 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.n_hot_cold = n_hot_cold;
     P.status = reinterpret_cast<int32_t*>(base + WsLayout::kStatus);
     P.ticket = reinterpret_cast<int32_t*>(base + WsLayout::kCounters);
+    P.next_unit = P.ticket + 1;
+    P.cold_tile = cold_token_tile(p);
+    P.cold_stages = std::min(kMaxStages, kTileBytes / (kABytes + P.cold_tile * 128));
+    const WsLayout L = ws_layout(p);
+    P.n_split = L.n_split;
+    P.part_done = reinterpret_cast<int32_t*>(base + L.part_done_off);
+    P.partials = reinterpret_cast<float*>(base + L.partials_off);
     P.ready = reinterpret_cast<int32_t*>(base + WsLayout::kTiles);
     P.trace = g_trace;
     P.trace_slots = g_trace_slots;
