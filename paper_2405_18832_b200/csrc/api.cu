@@ -86,11 +86,9 @@ int monde_route(const monde_problem* p, const void* x, const void* Wg, const flo
     if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
     if ((st = check_arch()) != MONDE_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (p->T > 0) {
-        st = launch_route(*p, x, Wg, bg, topk_idx, topk_w, probs, s);
-        if (st != MONDE_OK) return st;
-    }
-    return launch_histogram_classify_scan(*p, topk_idx, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold, s);
+    int32_t* ticket = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + WsLayout::kRouteTicket);
+    return launch_route(*p, x, Wg, bg, topk_idx, topk_w, probs, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold,
+                        ticket, s);
 }
 
 int monde_permute(const monde_problem* p, const void* x, const int32_t* topk_idx,

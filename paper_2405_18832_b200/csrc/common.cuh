@@ -17,6 +17,7 @@ constexpr int kMaxTopK = 8;
 // Workspace carving.  Offsets in bytes from the workspace base.
 struct WsLayout {
     static constexpr size_t kStatus = 0;        // int32 status, int32 site
+    static constexpr size_t kRouteTicket = 512; // int32: router CTAs finished
     static constexpr size_t kCounters = 1024;   // int32 counters used by the FFN kernels
     static constexpr size_t kCountersBytes = 15 * 1024;
     static constexpr size_t kTiles = 16 * 1024; // work lists built on the device
@@ -120,11 +121,11 @@ __device__ __forceinline__ float apply_act(float v, int act) {
 }
 
 // ---- launch prototypes (each returns a monde_status) -------------------------
+// Gate + softmax + top-k; the router CTA that finishes last also runs the histogram,
+// classification and scan.  `ticket` is an int32 in the workspace header (zero between calls).
 int launch_route(const monde_problem& p, const void* x, const void* Wg, const float* bg,
-                 int32_t* topk_idx, float* topk_w, float* probs, cudaStream_t s);
-int launch_histogram_classify_scan(const monde_problem& p, const int32_t* topk_idx, int32_t* counts,
-                                   int32_t* offsets, uint8_t* cls, int32_t* hot_ids, int32_t* cold_ids,
-                                   int32_t* n_hot_cold, cudaStream_t s);
+                 int32_t* topk_idx, float* topk_w, float* probs, int32_t* counts, int32_t* offsets, uint8_t* cls,
+                 int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, int32_t* ticket, cudaStream_t s);
 int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_idx, const int32_t* offsets,
                    int32_t* perm, int32_t* inv_perm, void* x_perm, cudaStream_t s);
 int launch_combine(const monde_problem& p, const void* y_perm, const int32_t* inv_perm,

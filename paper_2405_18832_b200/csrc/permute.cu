@@ -8,12 +8,15 @@ namespace monde {
 
 namespace {
 
-constexpr int kChunk = 32;           // assignments per CTA: one warp ranks them
-constexpr int kThreads = 128;        // all four warps copy rows
+constexpr int kChunk = 16;           // assignments per CTA, ranked by half a warp
+constexpr int kThreads = 128;        // four warps, four rows each
+constexpr int kRowsPerWarp = kChunk / (kThreads / 32);
 
 // CTA c owns assignments [c*kChunk, (c+1)*kChunk).  The number of earlier assignments to
 // each expert is recounted from topk_idx (at most A integers, L2-resident), which keeps
-// the kernel single-pass and free of inter-CTA ordering.
+// the kernel single-pass and free of inter-CTA ordering.  Small chunks give many CTAs and
+// every warp keeps the loads of its four rows in flight together, which is what matters
+// for a decode-sized batch where the whole gather is a few dozen rows.
 template <typename T>
 __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
         int A, int E, int k, int d, const T* __restrict__ x, const int32_t* __restrict__ topk_idx,
@@ -29,7 +32,7 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
     __syncthreads();
     if (warp == 0) {
         const int a = first + lane;
-        const int e = a < A ? topk_idx[a] : -1;
+        const int e = (lane < kChunk && a < A) ? topk_idx[a] : -1;
         const unsigned same = __match_any_sync(0xffffffffu, e);
         int pos = -1;
         if (e >= 0) {
@@ -37,18 +40,29 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
             perm[pos] = a;
             inv_perm[a] = pos;
         }
-        row_pos[lane] = pos;
+        if (lane < kChunk) row_pos[lane] = pos;
     }
     __syncthreads();
-    // Row gather: each warp copies whole rows with 16-byte accesses.
+    // Row gather with 16-byte accesses; the warp's rows advance together.
     constexpr int V = Vec16<T>::N;
     const int vec_per_row = d / V;
-    for (int r = warp; r < kChunk; r += kThreads / 32) {
-        const int p = row_pos[r];
-        if (p < 0) break;
-        const uint4* src = reinterpret_cast<const uint4*>(x + static_cast<int64_t>((first + r) / k) * d);
-        uint4* dst = reinterpret_cast<uint4*>(x_perm + static_cast<int64_t>(p) * d);
-        for (int i = lane; i < vec_per_row; i += 32) dst[i] = src[i];
+    const uint4* src[kRowsPerWarp];
+    uint4* dst[kRowsPerWarp];
+#pragma unroll
+    for (int r = 0; r < kRowsPerWarp; ++r) {
+        const int idx = warp * kRowsPerWarp + r;
+        const int p = row_pos[idx];
+        src[r] = p >= 0 ? reinterpret_cast<const uint4*>(x + static_cast<int64_t>((first + idx) / k) * d) : nullptr;
+        dst[r] = p >= 0 ? reinterpret_cast<uint4*>(x_perm + static_cast<int64_t>(p) * d) : nullptr;
+    }
+    for (int i = lane; i < vec_per_row; i += 32) {
+        uint4 v[kRowsPerWarp];
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r)
+            if (src[r] != nullptr) v[r] = src[r][i];
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r)
+            if (dst[r] != nullptr) dst[r][i] = v[r];
     }
 }
 

@@ -86,16 +86,99 @@ __device__ __forceinline__ void softmax_topk_store(const float (&logit)[kSlots],
     }
 }
 
+struct HistArgs {
+    int A, E, theta;
+    int32_t* counts;
+    int32_t* offsets;
+    uint8_t* cls;
+    int32_t* hot_ids;
+    int32_t* cold_ids;
+    int32_t* n_hot_cold;
+    int32_t* ticket;      // CTAs of the router that have finished (left at zero)
+};
+
+// Histogram of assignments per expert (shared-memory atomics on integers: the sum does
+// not depend on order), then classification, compaction and exclusive scan by one warp.
+// Runs in one CTA of any size.
+__device__ void histogram_classify_scan(const HistArgs& h, const int32_t* __restrict__ topk_idx, int* hist) {
+    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) hist[e] = 0;
+    __syncthreads();
+    for (int a = threadIdx.x; a < h.A; a += blockDim.x) atomicAdd(&hist[__ldcg(topk_idx + a)], 1);
+    __syncthreads();
+    if (threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
+    // lane owns experts [lane*8, lane*8+8)
+    int c[kSlots], sum = 0, nh = 0, nc = 0;
+#pragma unroll
+    for (int i = 0; i < kSlots; ++i) {
+        const int e = lane * kSlots + i;
+        c[i] = e < h.E ? hist[e] : 0;
+        sum += c[i];
+        nh += (c[i] > 0 && c[i] >= h.theta);
+        nc += (c[i] > 0 && c[i] < h.theta);
+    }
+    int ps = sum, ph = nh, pc = nc;   // inclusive scans across lanes
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, ps, o);
+        const int b = __shfl_up_sync(0xffffffffu, ph, o);
+        const int d = __shfl_up_sync(0xffffffffu, pc, o);
+        if (lane >= o) { ps += a; ph += b; pc += d; }
+    }
+    int off = ps - sum, ih = ph - nh, ic = pc - nc;
+#pragma unroll
+    for (int i = 0; i < kSlots; ++i) {
+        const int e = lane * kSlots + i;
+        if (e < h.E) {
+            h.counts[e] = c[i];
+            h.offsets[e] = off;
+            uint8_t k = 0;
+            if (c[i] > 0) {
+                if (c[i] >= h.theta) { k = 2; h.hot_ids[ih++] = e; }
+                else { k = 1; h.cold_ids[ic++] = e; }
+            }
+            h.cls[e] = k;
+            off += c[i];
+        }
+    }
+    if (lane == 31) {
+        h.offsets[h.E] = ps;
+        h.n_hot_cold[0] = ph;
+        h.n_hot_cold[1] = pc;
+    }
+}
+
+// Called by every thread of every router CTA after its top-k stores: the CTA that finishes
+// last runs the histogram, so routing is one launch.
+__device__ void finish_route(const HistArgs& h, const int32_t* topk_idx) {
+    __shared__ int s_hist[kMaxExperts];
+    __shared__ int s_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(h.ticket, 1) == static_cast<int>(gridDim.x) - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) *h.ticket = 0;
+    histogram_classify_scan(h, topk_idx, s_hist);
+}
+
+// Stand-alone form, used when there are no tokens (every count is zero).
+__global__ void __launch_bounds__(256) histogram_only_kernel(HistArgs h, const int32_t* topk_idx) {
+    __shared__ int s_hist[kMaxExperts];
+    histogram_classify_scan(h, topk_idx, s_hist);
+}
+
 // One warp per token; lanes split d_model with 16-byte loads.
 template <typename T>
 __global__ void __launch_bounds__(128) route_warp_per_token_kernel(
         int T_tokens, int d, int E, int k, int renorm, const T* __restrict__ x, const T* __restrict__ Wg,
         const float* __restrict__ bg, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
-        float* __restrict__ probs) {
+        float* __restrict__ probs, const HistArgs hist) {
     constexpr int V = Vec16<T>::N;
     const int lane = threadIdx.x & 31;
     const int64_t t = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (t >= T_tokens) return;
+    if (t < T_tokens) {
     const T* xr = x + t * d;
     float logit[kSlots];
 #pragma unroll
@@ -121,8 +204,9 @@ __global__ void __launch_bounds__(128) route_warp_per_token_kernel(
         }
     }
     softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs);
+    }
+    finish_route(hist, topk_idx);
 }
-
 
 // ---- bf16 gate on the warp-level tensor-core path -------------------------------------
 // CTA = 16 tokens x all experts; each of the 4 warps owns a contiguous quarter of the
@@ -140,13 +224,17 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 }
 
 template <int kTilesPerWarp>   // 8-expert column tiles per warp: padded E = 32 * kTilesPerWarp
-__global__ void __launch_bounds__(128) route_mma_kernel(
+__global__ void __launch_bounds__(512) route_mma_kernel(
         int T_tokens, int d, int E, int k, int renorm, const __nv_bfloat16* __restrict__ x,
         const __nv_bfloat16* __restrict__ Wg, const float* __restrict__ bg, int32_t* __restrict__ topk_idx,
-        float* __restrict__ topk_w, float* __restrict__ probs) {
+        float* __restrict__ topk_w, float* __restrict__ probs, const HistArgs hist) {
+    // 16 warps = 4 expert quarters x 4 interleaved K quarters: many independent loads in flight
+    // per CTA, which is what a 32-token decode batch (two CTAs in the whole grid) needs.
     constexpr int kEPad = 32 * kTilesPerWarp;
-    __shared__ float s_logit[16][kEPad + 1];
+    constexpr int kRow = kEPad + 1;
+    extern __shared__ float s_part[];                 // [4 K quarters][16 tokens][kRow]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int eq = warp & 3, kq = warp >> 2;
     const int g = lane >> 2, t4 = lane & 3;
     const int tok0 = blockIdx.x * 16;
     const int r0 = min(tok0 + g, T_tokens - 1), r1 = min(tok0 + g + 8, T_tokens - 1);
@@ -155,7 +243,7 @@ __global__ void __launch_bounds__(128) route_mma_kernel(
     const uint4* wp[kTilesPerWarp];
 #pragma unroll
     for (int j = 0; j < kTilesPerWarp; ++j) {
-        const int e = min(warp * (8 * kTilesPerWarp) + j * 8 + g, E - 1);
+        const int e = min(eq * (8 * kTilesPerWarp) + j * 8 + g, E - 1);
         wp[j] = reinterpret_cast<const uint4*>(Wg + static_cast<int64_t>(e) * d) + t4;
     }
     float acc[kTilesPerWarp][4];
@@ -164,8 +252,8 @@ __global__ void __launch_bounds__(128) route_mma_kernel(
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[j][i] = 0.0f;
     const int steps = d / 32;               // 32 k per step: 4 lanes x 8 elements
-#pragma unroll 2
-    for (int s = 0; s < steps; ++s) {
+#pragma unroll 4
+    for (int s = kq; s < steps; s += 4) {
         const uint4 a = xa[s * 4], b = xb[s * 4];
 #pragma unroll
         for (int j = 0; j < kTilesPerWarp; ++j) {
@@ -174,115 +262,72 @@ __global__ void __launch_bounds__(128) route_mma_kernel(
             mma_bf16_16816(acc[j], a.z, b.z, a.w, b.w, w.z, w.w);
         }
     }
+    float* part = s_part + kq * (16 * kRow);
 #pragma unroll
     for (int j = 0; j < kTilesPerWarp; ++j) {
-        const int e = warp * (8 * kTilesPerWarp) + j * 8 + t4 * 2;
-        const float b0 = (bg != nullptr && e < E) ? bg[e] : 0.0f;
-        const float b1 = (bg != nullptr && e + 1 < E) ? bg[e + 1] : 0.0f;
-        s_logit[g][e] = acc[j][0] + b0;
-        s_logit[g][e + 1] = acc[j][1] + b1;
-        s_logit[g + 8][e] = acc[j][2] + b0;
-        s_logit[g + 8][e + 1] = acc[j][3] + b1;
+        const int e = eq * (8 * kTilesPerWarp) + j * 8 + t4 * 2;
+        part[g * kRow + e] = acc[j][0];
+        part[g * kRow + e + 1] = acc[j][1];
+        part[(g + 8) * kRow + e] = acc[j][2];
+        part[(g + 8) * kRow + e + 1] = acc[j][3];
     }
     __syncthreads();
-    for (int r = warp; r < 16; r += 4) {
-        const int64_t t = tok0 + r;
-        if (t >= T_tokens) break;
+    const int64_t t = tok0 + warp;          // one warp per token for softmax and top-k
+    if (t < T_tokens) {
         float logit[kSlots];
 #pragma unroll
         for (int s = 0; s < kSlots; ++s) {
             const int e = s * 32 + lane;
-            logit[s] = (s < kTilesPerWarp && e < E) ? s_logit[r][e] : -INFINITY;
+            if (s < kTilesPerWarp && e < E) {
+                const float* p = s_part + warp * kRow + e;    // K quarters summed in a fixed order
+                logit[s] = ((p[0] + p[16 * kRow]) + (p[32 * kRow] + p[48 * kRow])) + (bg != nullptr ? bg[e] : 0.0f);
+            } else {
+                logit[s] = -INFINITY;
+            }
         }
         softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs);
     }
+    finish_route(hist, topk_idx);
 }
 
 template <int kTilesPerWarp>
-void launch_route_mma(const monde_problem& p, const void* x, const void* Wg, const float* bg, int32_t* topk_idx,
-                      float* topk_w, float* probs, cudaStream_t s) {
-    route_mma_kernel<kTilesPerWarp><<<(p.T + 15) / 16, 128, 0, s>>>(
+int launch_route_mma(const monde_problem& p, const void* x, const void* Wg, const float* bg, int32_t* topk_idx,
+                     float* topk_w, float* probs, const HistArgs& hist, cudaStream_t s) {
+    constexpr int kSmem = 4 * 16 * (32 * kTilesPerWarp + 1) * 4;
+    if (kSmem > 48 * 1024) {
+        static const cudaError_t attr = cudaFuncSetAttribute(route_mma_kernel<kTilesPerWarp>,
+                                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        if (attr != cudaSuccess) return MONDE_ERR_CUDA;
+    }
+    route_mma_kernel<kTilesPerWarp><<<(p.T + 15) / 16, 512, kSmem, s>>>(
         p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),
-        static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs);
-}
-
-// Histogram of assignments per expert (shared-memory atomics on integers: the sum does
-// not depend on order), then classification, compaction and exclusive scan by one warp.
-__global__ void __launch_bounds__(1024) histogram_classify_scan_kernel(
-        int A, int E, int theta, const int32_t* __restrict__ topk_idx, int32_t* __restrict__ counts,
-        int32_t* __restrict__ offsets, uint8_t* __restrict__ cls, int32_t* __restrict__ hot_ids,
-        int32_t* __restrict__ cold_ids, int32_t* __restrict__ n_hot_cold) {
-    __shared__ int hist[kMaxExperts];
-    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) hist[e] = 0;
-    __syncthreads();
-    for (int a = threadIdx.x; a < A; a += blockDim.x) atomicAdd(&hist[topk_idx[a]], 1);
-    __syncthreads();
-    if (threadIdx.x >= 32) return;
-    const int lane = threadIdx.x;
-    // lane owns experts [lane*8, lane*8+8)
-    int c[kSlots], sum = 0, nh = 0, nc = 0;
-#pragma unroll
-    for (int i = 0; i < kSlots; ++i) {
-        const int e = lane * kSlots + i;
-        c[i] = e < E ? hist[e] : 0;
-        sum += c[i];
-        nh += (c[i] > 0 && c[i] >= theta);
-        nc += (c[i] > 0 && c[i] < theta);
-    }
-    int ps = sum, ph = nh, pc = nc;   // inclusive scans across lanes
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int a = __shfl_up_sync(0xffffffffu, ps, o);
-        const int b = __shfl_up_sync(0xffffffffu, ph, o);
-        const int d = __shfl_up_sync(0xffffffffu, pc, o);
-        if (lane >= o) { ps += a; ph += b; pc += d; }
-    }
-    int off = ps - sum, ih = ph - nh, ic = pc - nc;
-#pragma unroll
-    for (int i = 0; i < kSlots; ++i) {
-        const int e = lane * kSlots + i;
-        if (e < E) {
-            counts[e] = c[i];
-            offsets[e] = off;
-            uint8_t k = 0;
-            if (c[i] > 0) {
-                if (c[i] >= theta) { k = 2; hot_ids[ih++] = e; }
-                else { k = 1; cold_ids[ic++] = e; }
-            }
-            cls[e] = k;
-            off += c[i];
-        }
-    }
-    if (lane == 31) {
-        offsets[E] = ps;
-        n_hot_cold[0] = ph;
-        n_hot_cold[1] = pc;
-    }
+        static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs, hist);
+    return MONDE_OK;
 }
 
 }  // namespace
 
 int launch_route(const monde_problem& p, const void* x, const void* Wg, const float* bg,
-                 int32_t* topk_idx, float* topk_w, float* probs, cudaStream_t s) {
-    const int warps = 4;
-    const int grid = (p.T + warps - 1) / warps;
+                 int32_t* topk_idx, float* topk_w, float* probs, int32_t* counts, int32_t* offsets, uint8_t* cls,
+                 int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, int32_t* ticket, cudaStream_t s) {
+    const HistArgs hist{p.T * p.top_k, p.E, p.hot_threshold, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold, ticket};
+    if (p.T == 0) {
+        histogram_only_kernel<<<1, 256, 0, s>>>(hist, topk_idx);
+        return launched();
+    }
     if (p.dtype == MONDE_BF16) {
-        if (p.E <= 32) launch_route_mma<1>(p, x, Wg, bg, topk_idx, topk_w, probs, s);
-        else if (p.E <= 64) launch_route_mma<2>(p, x, Wg, bg, topk_idx, topk_w, probs, s);
-        else if (p.E <= 128) launch_route_mma<4>(p, x, Wg, bg, topk_idx, topk_w, probs, s);
-        else launch_route_mma<8>(p, x, Wg, bg, topk_idx, topk_w, probs, s);
-    } else
-        route_warp_per_token_kernel<float><<<grid, warps * 32, 0, s>>>(
+        int st;
+        if (p.E <= 32) st = launch_route_mma<1>(p, x, Wg, bg, topk_idx, topk_w, probs, hist, s);
+        else if (p.E <= 64) st = launch_route_mma<2>(p, x, Wg, bg, topk_idx, topk_w, probs, hist, s);
+        else if (p.E <= 128) st = launch_route_mma<4>(p, x, Wg, bg, topk_idx, topk_w, probs, hist, s);
+        else st = launch_route_mma<8>(p, x, Wg, bg, topk_idx, topk_w, probs, hist, s);
+        if (st != MONDE_OK) return st;
+    } else {
+        const int warps = 4;
+        route_warp_per_token_kernel<float><<<(p.T + warps - 1) / warps, warps * 32, 0, s>>>(
             p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const float*>(x),
-            static_cast<const float*>(Wg), bg, topk_idx, topk_w, probs);
-    return launched();
-}
-
-int launch_histogram_classify_scan(const monde_problem& p, const int32_t* topk_idx, int32_t* counts,
-                                   int32_t* offsets, uint8_t* cls, int32_t* hot_ids, int32_t* cold_ids,
-                                   int32_t* n_hot_cold, cudaStream_t s) {
-    histogram_classify_scan_kernel<<<1, 1024, 0, s>>>(p.T * p.top_k, p.E, p.hot_threshold, topk_idx, counts,
-                                                      offsets, cls, hot_ids, cold_ids, n_hot_cold);
+            static_cast<const float*>(Wg), bg, topk_idx, topk_w, probs, hist);
+    }
     return launched();
 }
 
