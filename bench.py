@@ -40,8 +40,8 @@ METRIC = "moe_ffn_layer_tokens_per_s"
 UNIT = "tokens/s"
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures
-# summarised under profiles/ (None until a capture exists for that workload).
-NCU_TRAFFIC_BYTES = {"C1": None, "C2": None, "C3": None}
+# summarised in profiles/expert_ffn_kernel_C1_C2.md (None where no capture exists).
+NCU_TRAFFIC_BYTES = {"C1": 620.6e6, "C2": 458.0e6, "C3": None}
 
 
 def measured_peaks():

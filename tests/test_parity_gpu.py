@@ -101,3 +101,33 @@ def test_results_are_bit_reproducible_and_threshold_independent():
         c = P.run_gpu(q, dev)
         assert torch.equal(a.perm, c.perm)
         P.check_close("out vs other class", P.widen(c.out), P.widen(a.out), "bf16")
+
+
+# ---- crossover sweep (E=64, top-2, d_ff = 4 d_model, GELU, renormalised weights) -------------
+# Expert outputs do not depend on the threshold, so each (d_model, T, alpha) point is computed once
+# by the oracle on a token sample and compared with the CUDA path at all three thresholds.
+
+@pytest.mark.parametrize("d_model,n_sample", [(1024, 24), (2048, 12), (4096, 6)])
+def test_crossover_sweep_sampled_parity(d_model, n_sample):
+    import dataclasses
+    weights = None
+    for T in (1, 8, 64, 512, 4096):
+        for alpha in (0.0, 1.2):
+            w = S.sweep_point(d_model, T, alpha, 16)
+            g = S.generate(w, with_weights=False)
+            dev = P.to_device(g)
+            if weights is None:      # same seed and tensor ids at every point of this d_model
+                gw = S.generate(w, weights_device="cuda")
+                weights = {k: gw[k] for k in ("W1", "W2", "b1", "b2")}
+            dev.update(weights)
+            ref = None
+            for theta in (4, 16, 64):
+                wt = dataclasses.replace(w, problem=dataclasses.replace(w.problem, hot_threshold=theta))
+                if ref is None:
+                    ref = P.check_sampled(wt, g, dev, n_tokens=n_sample)
+                    first = ref.buf
+                else:
+                    buf = P.run_gpu(wt.problem, dev, want_probs=False)
+                    P.check_routing(wt.problem, g, buf)
+                    # same experts, same rows: only the class, hence the tiling, may differ
+                    P.check_close(f"out theta={theta}", P.widen(buf.out), P.widen(first.out), "bf16")
