@@ -148,6 +148,31 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
 void count_launches(int n);
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? MONDE_OK : MONDE_ERR_CUDA; }
+
+// Programmatic dependent launch.  Every kernel of the library is launched with the
+// programmatic-stream-serialization attribute, calls pdl_launch_dependents() early (the next
+// kernel in the stream may then be scheduled and run its set-up), and calls pdl_wait() before
+// it reads anything another kernel may have produced and before it writes anything to global
+// memory.  pdl_wait() returns once the preceding kernel in the stream has completed and its
+// writes are visible; since that kernel waited the same way, everything earlier is complete too.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 inline int launched(int n = 1) {
     count_launches(n);
     return cuda_status(cudaGetLastError());

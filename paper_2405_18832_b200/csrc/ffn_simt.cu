@@ -17,6 +17,8 @@ __global__ void __launch_bounds__(kWarps * 32) linear_simt_kernel(
         int act, int K, int N, const T* __restrict__ in, const T* __restrict__ W, const T* __restrict__ bias,
         const int32_t* __restrict__ offsets, const int32_t* __restrict__ ids, const int32_t* __restrict__ n_ids,
         T* __restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
     if (static_cast<int>(blockIdx.y) >= *n_ids) return;
     constexpr int V = Vec16<T>::N;
     const int e = ids[blockIdx.y];
@@ -66,11 +68,11 @@ int launch_linear_simt(int dtype, int act_or_neg1, int E, int K, int N, const vo
                        void* out, cudaStream_t s) {
     dim3 grid((N + kWarps - 1) / kWarps, E);
     if (dtype == MONDE_BF16)
-        linear_simt_kernel<__nv_bfloat16><<<grid, kWarps * 32, 0, s>>>(
+        launch_pdl(linear_simt_kernel<__nv_bfloat16>, grid, dim3(kWarps * 32), 0, s,
             act_or_neg1, K, N, static_cast<const __nv_bfloat16*>(in), static_cast<const __nv_bfloat16*>(W),
             static_cast<const __nv_bfloat16*>(bias), offsets, ids, n_ids, static_cast<__nv_bfloat16*>(out));
     else
-        linear_simt_kernel<float><<<grid, kWarps * 32, 0, s>>>(
+        launch_pdl(linear_simt_kernel<float>, grid, dim3(kWarps * 32), 0, s,
             act_or_neg1, K, N, static_cast<const float*>(in), static_cast<const float*>(W),
             static_cast<const float*>(bias), offsets, ids, n_ids, static_cast<float*>(out));
     return launched();

@@ -34,6 +34,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -231,27 +232,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     auto q_empty = [&](int s) { return bar0 + 8u * (2 * kMaxStages + 6 + kQueue + s); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    ut.n_hot = min(P.n_hot_cold[0], kMaxExperts);
-    ut.n_all = min(ut.n_hot + P.n_hot_cold[1], kMaxExperts);
-    ut.nt1 = (P.d_ff + kTileRows - 1) / kTileRows;
-    ut.nt2 = (P.d_model + kTileRows - 1) / kTileRows;
 
-    // ---- set-up: unit table, barriers, tensor memory --------------------------------
-    for (int i = tid; i < ut.n_all; i += kThreads) {
-        const bool cold = i >= ut.n_hot;
-        const int e = cold ? P.cold_ids[i - ut.n_hot] : P.hot_ids[i];
-        const int tile = cold ? P.cold_tile : kHotTokTile;
-        const int m = P.counts[e];
-        const int tt = max(1, (m + tile - 1) / tile);
-        ut.e[i] = e;
-        ut.off[i] = P.offsets[e];
-        ut.m[i] = m;
-        ut.tt[i] = tt;
-        ut.per[i] = ((m + tt - 1) / tt + 15) & ~15;
-        ut.tt_prefix[i + 1] = tt;
-    }
+    // ---- set-up that touches nothing another kernel produced: runs while the preceding
+    // kernel of the stream is still finishing --------------------------------------------
+    pdl_launch_dependents();
     if (tid == 0) {
-        ut.tt_prefix[0] = 0;
         *abort_flag = 0;
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(full_bar(s), 1);    // producer's expect_tx arrival
@@ -267,7 +252,35 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             mbar_init(q_empty(s), 6);       // MMA issuer, 4 epilogue warps, publisher
         }
         fence_barrier_init();
+        prefetch_tensormap(&map_w1);
+        prefetch_tensormap(&map_w2);
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_h);
+    } else if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
     }
+    pdl_wait();
+
+    // ---- unit table from the router's outputs -----------------------------------------------
+    ut.n_hot = min(P.n_hot_cold[0], kMaxExperts);
+    ut.n_all = min(ut.n_hot + P.n_hot_cold[1], kMaxExperts);
+    ut.nt1 = (P.d_ff + kTileRows - 1) / kTileRows;
+    ut.nt2 = (P.d_model + kTileRows - 1) / kTileRows;
+    for (int i = tid; i < ut.n_all; i += kThreads) {
+        const bool cold = i >= ut.n_hot;
+        const int e = cold ? P.cold_ids[i - ut.n_hot] : P.hot_ids[i];
+        const int tile = cold ? P.cold_tile : kHotTokTile;
+        const int m = P.counts[e];
+        const int tt = max(1, (m + tile - 1) / tile);
+        ut.e[i] = e;
+        ut.off[i] = P.offsets[e];
+        ut.m[i] = m;
+        ut.tt[i] = tt;
+        ut.per[i] = ((m + tt - 1) / tt + 15) & ~15;
+        ut.tt_prefix[i + 1] = tt;
+    }
+    if (tid == 0) ut.tt_prefix[0] = 0;
     __syncthreads();
     if (warp == 0) {   // inclusive scan of the per-expert token-tile counts, 8 entries per lane
         int v[8], sum = 0;
@@ -290,9 +303,6 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             run += v[i];
             if (idx < ut.n_all) ut.tt_prefix[idx + 1] = run;
         }
-    } else if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-        tmem_relinquish();
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -328,10 +338,6 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     if (warp == 0) {
         // ---- scheduler + TMA producer ------------------------------------------------------
         if (lane == 0) {
-            prefetch_tensormap(&map_w1);
-            prefetch_tensormap(&map_w2);
-            prefetch_tensormap(&map_x);
-            prefetch_tensormap(&map_h);
             const uint64_t pol_w = policy_evict_first();   // weights are read once
             const uint64_t pol_x = policy_evict_last();    // token tiles are re-read by every feature tile
             int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes;
@@ -653,8 +659,9 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, ui
     const cuuint64_t strides[1] = {cols * 2};
     const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
     const cuuint32_t estr[2] = {1, 1};
+    static const int promo = [] { const char* e = getenv("MONDE_L2PROMO"); return e ? atoi(e) : 3; }();
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, static_cast<CUtensorMapL2promotion>(promo),
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -716,10 +723,14 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     if (!make_map(&map_w2, W2, static_cast<uint64_t>(p.E) * p.d_model, p.d_ff, kTileRows)) return MONDE_ERR_CUDA;
     if (!make_map(&map_x, x_perm, A, p.d_model, 16)) return MONDE_ERR_CUDA;
     if (!make_map(&map_h, P.h, A, p.d_ff, 16)) return MONDE_ERR_CUDA;
+    cudaError_t err;
     if (p.act == MONDE_ACT_RELU)
-        expert_ffn_kernel<MONDE_ACT_RELU><<<sm_count(), kThreads, kSmemBytes, s>>>(map_w1, map_w2, map_x, map_h, P);
+        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_RELU>, dim3(sm_count()), dim3(kThreads), kSmemBytes, s, map_w1,
+                         map_w2, map_x, map_h, P);
     else
-        expert_ffn_kernel<MONDE_ACT_GELU_ERF><<<sm_count(), kThreads, kSmemBytes, s>>>(map_w1, map_w2, map_x, map_h, P);
+        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_GELU_ERF>, dim3(sm_count()), dim3(kThreads), kSmemBytes, s,
+                         map_w1, map_w2, map_x, map_h, P);
+    if (err != cudaSuccess) return MONDE_ERR_CUDA;
     return launched();
 }
 

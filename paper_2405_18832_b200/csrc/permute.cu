@@ -26,8 +26,10 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
     __shared__ int row_pos[kChunk];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int first = blockIdx.x * kChunk;
+    pdl_launch_dependents();
     for (int e = tid; e < kMaxExperts; e += kThreads) before[e] = 0;
     __syncthreads();
+    pdl_wait();
     for (int a = tid; a < first; a += kThreads) atomicAdd(&before[topk_idx[a]], 1);
     __syncthreads();
     if (warp == 0) {
@@ -74,6 +76,8 @@ __global__ void __launch_bounds__(256) combine_kernel(
     constexpr int V = Vec16<T>::N;
     const int vec_per_row = d / V;
     const int64_t g = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     if (g >= static_cast<int64_t>(T_tokens) * vec_per_row) return;
     const int64_t t = g / vec_per_row;
     const int c = static_cast<int>(g % vec_per_row) * V;
@@ -98,11 +102,11 @@ int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_id
     const int A = p.T * p.top_k;
     const int grid = (A + kChunk - 1) / kChunk;
     if (p.dtype == MONDE_BF16)
-        permute_gather_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(
+        launch_pdl(permute_gather_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), 0, s,
             A, p.E, p.top_k, p.d_model, static_cast<const __nv_bfloat16*>(x), topk_idx, offsets, perm,
             inv_perm, static_cast<__nv_bfloat16*>(x_perm));
     else
-        permute_gather_kernel<float><<<grid, kThreads, 0, s>>>(
+        launch_pdl(permute_gather_kernel<float>, dim3(grid), dim3(kThreads), 0, s,
             A, p.E, p.top_k, p.d_model, static_cast<const float*>(x), topk_idx, offsets, perm, inv_perm,
             static_cast<float*>(x_perm));
     return launched();
@@ -114,11 +118,11 @@ int launch_combine(const monde_problem& p, const void* y_perm, const int32_t* in
     const int64_t n = static_cast<int64_t>(p.T) * (p.d_model / V);
     const int grid = static_cast<int>((n + 255) / 256);
     if (p.dtype == MONDE_BF16)
-        combine_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(
+        launch_pdl(combine_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, s,
             p.T, p.d_model, p.top_k, static_cast<const __nv_bfloat16*>(y_perm), inv_perm, topk_w,
             static_cast<__nv_bfloat16*>(out));
     else
-        combine_kernel<float><<<grid, 256, 0, s>>>(p.T, p.d_model, p.top_k, static_cast<const float*>(y_perm),
+        launch_pdl(combine_kernel<float>, dim3(grid), dim3(256), 0, s, p.T, p.d_model, p.top_k, static_cast<const float*>(y_perm),
                                                    inv_perm, topk_w, static_cast<float*>(out));
     return launched();
 }

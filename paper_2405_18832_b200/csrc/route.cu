@@ -166,6 +166,8 @@ __device__ void finish_route(const HistArgs& h, const int32_t* topk_idx) {
 // Stand-alone form, used when there are no tokens (every count is zero).
 __global__ void __launch_bounds__(256) histogram_only_kernel(HistArgs h, const int32_t* topk_idx) {
     __shared__ int s_hist[kMaxExperts];
+    pdl_launch_dependents();
+    pdl_wait();
     histogram_classify_scan(h, topk_idx, s_hist);
 }
 
@@ -178,6 +180,8 @@ __global__ void __launch_bounds__(128) route_warp_per_token_kernel(
     constexpr int V = Vec16<T>::N;
     const int lane = threadIdx.x & 31;
     const int64_t t = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    pdl_launch_dependents();
+    pdl_wait();
     if (t < T_tokens) {
     const T* xr = x + t * d;
     float logit[kSlots];
@@ -237,6 +241,8 @@ __global__ void __launch_bounds__(512) route_mma_kernel(
     const int eq = warp & 3, kq = warp >> 2;
     const int g = lane >> 2, t4 = lane & 3;
     const int tok0 = blockIdx.x * 16;
+    pdl_launch_dependents();
+    pdl_wait();
     const int r0 = min(tok0 + g, T_tokens - 1), r1 = min(tok0 + g + 8, T_tokens - 1);
     const uint4* xa = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(r0) * d) + t4;
     const uint4* xb = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(r1) * d) + t4;
@@ -299,7 +305,7 @@ int launch_route_mma(const monde_problem& p, const void* x, const void* Wg, cons
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (attr != cudaSuccess) return MONDE_ERR_CUDA;
     }
-    route_mma_kernel<kTilesPerWarp><<<(p.T + 15) / 16, 512, kSmem, s>>>(
+    launch_pdl(route_mma_kernel<kTilesPerWarp>, dim3((p.T + 15) / 16), dim3(512), kSmem, s,
         p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),
         static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs, hist);
     return MONDE_OK;
@@ -312,7 +318,7 @@ int launch_route(const monde_problem& p, const void* x, const void* Wg, const fl
                  int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, int32_t* ticket, cudaStream_t s) {
     const HistArgs hist{p.T * p.top_k, p.E, p.hot_threshold, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold, ticket};
     if (p.T == 0) {
-        histogram_only_kernel<<<1, 256, 0, s>>>(hist, topk_idx);
+        launch_pdl(histogram_only_kernel, dim3(1), dim3(256), 0, s, hist, topk_idx);
         return launched();
     }
     if (p.dtype == MONDE_BF16) {
@@ -324,7 +330,7 @@ int launch_route(const monde_problem& p, const void* x, const void* Wg, const fl
         if (st != MONDE_OK) return st;
     } else {
         const int warps = 4;
-        route_warp_per_token_kernel<float><<<(p.T + warps - 1) / warps, warps * 32, 0, s>>>(
+        launch_pdl(route_warp_per_token_kernel<float>, dim3((p.T + warps - 1) / warps), dim3(warps * 32), 0, s,
             p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const float*>(x),
             static_cast<const float*>(Wg), bg, topk_idx, topk_w, probs, hist);
     }
