@@ -146,6 +146,39 @@ int monde_combine(const monde_problem* p, const void* y_perm, const int32_t* inv
  * receives an implementation-defined code saying which wait gave up. */
 int monde_poll_device_status(void* ws, void* stream, int32_t* site);
 
+/* monde_moe_ffn_fwd for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, same arithmetic, same outputs.)
+ *
+ * Who needs it: a serving loop that allocates everything at start-up and forbids cudaMalloc
+ * afterwards, a plug-in that is handed its input and output buffers and owns no allocator,
+ * code that runs where growing a memory pool is not allowed.  Such a caller has nowhere to
+ * get the workspace that monde_moe_ffn_fwd asks for, so this entry point uses a fixed
+ * scratch array of MONDE_STATIC_WS_BYTES that is part of the library's device image.  The
+ * call itself allocates and frees nothing.
+ *
+ *  - Arguments are those of monde_moe_ffn_fwd without ws / ws_bytes; inputs and outputs are
+ *    still the caller's device buffers.
+ *  - Limit: monde_workspace_bytes(p) must not exceed MONDE_STATIC_WS_BYTES; otherwise the call
+ *    returns MONDE_ERR_WORKSPACE and launches nothing.  (Decode-sized batches fit: E=128,
+ *    d_model=1024, d_ff=4096, T=32 needs about 26 MB; a 4096-token batch does not.)
+ *  - Every GPU that loads the library holds the array from load until the process exits.
+ *  - The first call on a device looks up the array's device address (once per device, with
+ *    that device current).  Make that first call before any stream capture begins.
+ *  - All calls on a GPU share the one array, and it keeps the previous call's contents; the
+ *    entry point clears the parts that must start at zero (in stream order) before it
+ *    launches.  Two calls that overlap on the GPU - different streams, or the same stream
+ *    from two threads without ordering - race on the array and give undefined results:
+ *    order them, or use monde_moe_ffn_fwd with separate workspaces.
+ *  - After MONDE_ERR_TIMEOUT from a previous call nothing special is needed: the next call
+ *    clears the header again.  monde_poll_device_status does not apply (no caller-visible ws).
+ */
+#define MONDE_STATIC_WS_BYTES (32u << 20)
+int monde_moe_ffn_fwd_static_ws(const monde_problem* p, const void* x_perm,
+                                const void* W1, const void* b1, const void* W2, const void* b2,
+                                const int32_t* counts, const int32_t* offsets, const uint8_t* cls,
+                                const int32_t* hot_ids, const int32_t* cold_ids, const int32_t* n_hot_cold,
+                                void* y_perm, void* stream);
+
 /* Diagnostic: number of kernels this library has launched in this process so far. */
 long long monde_kernel_launches(void);
 

@@ -17,7 +17,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmonde.so")
 
 SYMBOLS = ("monde_workspace_bytes", "monde_status_string", "monde_route", "monde_permute",
-           "monde_moe_ffn_fwd", "monde_combine", "monde_poll_device_status", "monde_kernel_launches")
+           "monde_moe_ffn_fwd", "monde_moe_ffn_fwd_static_ws", "monde_combine", "monde_poll_device_status",
+           "monde_kernel_launches")
 
 _DTYPE = {"f32": 0, "bf16": 1}
 _ACT = {"relu": 0, "gelu": 1}
@@ -60,6 +61,8 @@ def lib() -> ctypes.CDLL:
         L.monde_moe_ffn_fwd.restype = ctypes.c_int
         L.monde_moe_ffn_fwd.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, i32p, i32p, i32p, vp,
                                         vp, ctypes.c_size_t, vp]
+        L.monde_moe_ffn_fwd_static_ws.restype = ctypes.c_int
+        L.monde_moe_ffn_fwd_static_ws.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, i32p, i32p, i32p, vp, vp]
         L.monde_combine.restype = ctypes.c_int
         L.monde_combine.argtypes = [pp, vp, i32p, f32p, vp, vp]
         L.monde_poll_device_status.restype = ctypes.c_int
@@ -123,6 +126,21 @@ def monde_moe_ffn_fwd(p, x_perm, W1, b1, W2, b2, counts, offsets, cls, hot_ids, 
         ctypes.byref(cp), _ptr(x_perm), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(counts), _ptr(offsets),
         _ptr(cls), _ptr(hot_ids), _ptr(cold_ids), _ptr(n_hot_cold), _ptr(y_perm),
         _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+STATIC_WS_BYTES = 32 << 20
+
+
+def monde_moe_ffn_fwd_static_ws(p, x_perm, W1, b1, W2, b2, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold,
+                                y_perm, stream=None) -> None:
+    """Expert FFN without a caller workspace, for callers that may not allocate device memory
+    (pre-allocated serving loops, plug-ins without an allocator): the scratch is a fixed
+    array inside the library, shared by all calls on the GPU, so calls must not overlap.
+    Raises MondeError(workspace too small) when the problem needs more than STATIC_WS_BYTES."""
+    cp = c_problem(p)
+    _check("monde_moe_ffn_fwd_static_ws", lib().monde_moe_ffn_fwd_static_ws(
+        ctypes.byref(cp), _ptr(x_perm), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(counts), _ptr(offsets),
+        _ptr(cls), _ptr(hot_ids), _ptr(cold_ids), _ptr(n_hot_cold), _ptr(y_perm), _stream(stream)))
 
 
 def monde_combine(p, y_perm, inv_perm, topk_w, out, stream=None) -> None:
