@@ -60,7 +60,7 @@ constexpr int kTileBytes = 192 * 1024;
 constexpr int kNumBars = 2 * kMaxStages + 6 + 2 * kQueue;
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
 constexpr int kStageOutBytes = 2 * 16 * kTileRows * 2;
-constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kTableInts * 4 + kStageOutBytes + 16;
+constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kQueue * 64 + kTableInts * 4 + kStageOutBytes + 16;
 constexpr int kTmemCols = 512;        // two accumulator buffers of 256 fp32 columns
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
 
@@ -102,6 +102,7 @@ __device__ __forceinline__ void trace_time(const FfnParams& P, int it, int slot)
 }
 
 struct Unit {
+    int id;       // position in the unit list, -1 = end of list
     int e;        // expert id
     int row0;     // first row of the token tile in the expert-contiguous buffers
     int rows;     // valid token rows in the tile
@@ -115,6 +116,8 @@ struct Unit {
     int n_split;    // sub-units of this tile (1 unless cold second layer)
     int tile_idx;   // cold second-layer tile index (partials / part_done)
 };
+
+static_assert(sizeof(Unit) <= 64, "unit queue slots are 64 bytes");
 
 // Per-CTA copy of the unit list in shared memory.  Entries 0..n_hot-1 are the hot experts,
 // n_hot..n_hot+n_cold-1 the cold ones; tt_prefix is the exclusive prefix of token tiles.
@@ -132,6 +135,7 @@ struct UnitTable {
 
     __device__ __forceinline__ Unit decode(int u) const {
         Unit r;
+        r.id = u;
         int v;
         if (u < seg1) { r.cold = 0; r.layer = 0; v = u; }
         else if (u < seg2) { r.cold = 0; r.layer = 1; v = u - seg1; }
@@ -209,8 +213,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTileBytes);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    volatile int* unit_queue = reinterpret_cast<volatile int*>(tmem_slot + 4);      // [kQueue]
-    int* tab = reinterpret_cast<int*>(tmem_slot + 16);
+    int* unit_queue = reinterpret_cast<int*>(tmem_slot + 16);      // [kQueue] decoded units, 16 ints each
+    int* tab = unit_queue + kQueue * 16;
     __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(                     // 2 x [16 tokens][128 features]
         (reinterpret_cast<uintptr_t>(tab + kTableInts) + 15) & ~uintptr_t(15));
     UnitTable ut;
@@ -323,16 +327,22 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     const int cold_stage_bytes = kABytes + P.cold_tile * 128;
     const int hot_stage_bytes = kABytes + kHotTokTile * 128;
 
-    // Every role but the producer takes its next unit id from the shared-memory queue.
-    // Returns -1 at the end of the list or when a wait gave up.
-    // `whole_warp`: all 32 lanes call (epilogue warps); otherwise a single lane calls.
-    auto pop_unit = [&](int it, bool whole_warp) -> int {
+    // The producer decodes every unit once, one unit ahead of its loads, and hands the decoded
+    // record to the other roles through a small shared-memory queue (decoding costs about half
+    // a microsecond of dependent shared-memory loads and divisions: too much to repeat in every
+    // role at the start of every 6 us unit).  id = -1 marks the end of the list or a wait that
+    // gave up.  `whole_warp`: all 32 lanes call (epilogue warps); otherwise a single lane calls.
+    auto pop_unit = [&](int it, bool whole_warp) -> Unit {
         const int slot = it % kQueue;
-        if (!mbar_wait(q_full(slot), (it / kQueue) & 1, abort_flag, kWaitLimitNs)) return -1;
-        const int u = unit_queue[slot];
+        Unit un;
+        if (!mbar_wait(q_full(slot), (it / kQueue) & 1, abort_flag, kWaitLimitNs)) {
+            un.id = -1;
+            return un;
+        }
+        un = *reinterpret_cast<const Unit*>(unit_queue + slot * 16);
         if (whole_warp) __syncwarp();
         if (lane == 0) mbar_arrive(q_empty(slot));
-        return u;
+        return un;
     };
 
     if (warp == 0) {
@@ -343,21 +353,26 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes;
             uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
             bool ok = true;
-            int u_next = atomicAdd(P.next_unit, 1);     // one id ahead: hides the atomic's round trip
-            for (int it = 0; ok; ++it) {
-                const int slot = it % kQueue;
-                if (!mbar_wait(q_empty(slot), ((it / kQueue) & 1) ^ 1, abort_flag, kWaitLimitNs)) {
+            // Publishes unit number `j` of this CTA (or the end marker) to the other roles.
+            auto push_unit = [&](int j, const Unit& un) -> bool {
+                const int slot = j % kQueue;
+                if (!mbar_wait(q_empty(slot), ((j / kQueue) & 1) ^ 1, abort_flag, kWaitLimitNs)) {
                     report_timeout(P.status, abort_flag, kSiteQueue);
-                    break;
+                    return false;
                 }
-                int u = u_next;
-                if (u >= ut.total_units) u = -1;
-                else u_next = atomicAdd(P.next_unit, 1);
-                unit_queue[slot] = u;
-                mbar_arrive(q_full(slot));          // release: the id is visible to whoever acquires
-                if (u < 0) break;
-                const Unit un = ut.decode(u);
-                trace_mark(P, it, 0, static_cast<unsigned long long>(u));
+                *reinterpret_cast<Unit*>(unit_queue + slot * 16) = un;
+                mbar_arrive(q_full(slot));          // release: the record is visible to whoever acquires
+                return true;
+            };
+            Unit cur, nxt;
+            int u = atomicAdd(P.next_unit, 1);
+            cur.id = -1;
+            if (u < ut.total_units) cur = ut.decode(u);
+            ok = push_unit(0, cur);
+            int u_ahead = cur.id >= 0 ? atomicAdd(P.next_unit, 1) : 0;   // consumed a few K blocks later
+            for (int it = 0; ok && cur.id >= 0; ++it) {
+                const Unit un = cur;
+                trace_mark(P, it, 0, static_cast<unsigned long long>(un.id));
                 if (un.cold != cls) {
                     // geometry switch: every stage filled so far must have been consumed
                     for (int s = 0; ok && s < stages; ++s)
@@ -374,7 +389,18 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                 const CUtensorMap* mw = un.layer ? &map_w2 : &map_w1;
                 const CUtensorMap* mi = un.layer ? &map_h : &map_x;
                 const int N = un.layer ? P.d_model : P.d_ff;
+                bool next_ready = false;
                 for (int kb = un.kb0; kb < un.kb1; ++kb) {
+                    if (!next_ready && (kb - un.kb0 == 2 || kb == un.kb1 - 1)) {
+                        // take, decode and publish the next unit while this one's loads are in flight
+                        nxt.id = -1;
+                        if (u_ahead < ut.total_units) {
+                            nxt = ut.decode(u_ahead);
+                            u_ahead = atomicAdd(P.next_unit, 1);
+                        }
+                        if (!push_unit(it + 1, nxt)) { ok = false; break; }
+                        next_ready = true;
+                    }
                     if (!mbar_wait(empty_bar(stage), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteProducerEmpty);
                         ok = false;
@@ -407,6 +433,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     if (++stage == stages) stage = 0;
                 }
                 trace_time(P, it, 2);
+                cur = nxt;
             }
         }
     } else if (warp == 1) {
@@ -416,9 +443,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             uint32_t use_bits = 0;      // bit s: parity of the number of uses of stage s
             bool ok = true;
             for (int it = 0; ok; ++it) {
-                const int u = pop_unit(it, false);
-                if (u < 0) break;
-                const Unit un = ut.decode(u);
+                const Unit un = pop_unit(it, false);
+                if (un.id < 0) break;
                 if (un.cold != cls) {
                     cls = un.cold;
                     stages = cls ? P.cold_stages : kHotStages;
@@ -460,13 +486,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         // ---- epilogue: TMEM -> registers -> bias, activation -> shared -> global -------------
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         for (int it = 0;; ++it) {
-            const int u = pop_unit(it, true);
+            const Unit un = pop_unit(it, true);
             const int b = it & 1;
             const uint32_t tphase = (it >> 1) & 1;
-            bool got = u >= 0;
-            Unit un;
+            bool got = un.id >= 0;
             if (got) {
-                un = ut.decode(u);
                 got = mbar_wait(acc_full(b), tphase, abort_flag, kWaitLimitNs);
                 if (!got) report_timeout(P.status, abort_flag, kSiteEpilogueTmemFull);
             }
@@ -588,9 +612,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         // at CTA scope) -> this thread's device-scope fence (cumulative) -> counter increment.
         if (lane == 0) {
             for (int it = 0;; ++it) {
-                const int u = pop_unit(it, false);
-                if (u < 0) break;
-                const Unit un = ut.decode(u);
+                const Unit un = pop_unit(it, false);
+                if (un.id < 0) break;
                 const int b = it & 1;
                 if (!mbar_wait(rows_stored(b), (it >> 1) & 1, abort_flag, kWaitLimitNs))
                     break;   // the role that stalled has already reported
