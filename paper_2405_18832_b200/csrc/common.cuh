@@ -53,7 +53,7 @@ inline WsLayout ws_layout(const monde_problem& p) {
     // the partial tiles fit a bounded scratch (otherwise no split).
     const size_t ct = cold_token_tile(p);
     const size_t nt2 = (static_cast<size_t>(p.d_model) + 127) / 128;
-    const size_t cold_tiles = (A / ct + p.E) * nt2;          // upper bound on cold second-layer tiles
+    const size_t cold_tiles = (A / ct + p.E) * (nt2 + 1);    // upper bound on cold second-layer tiles (units cover pairs)
     int split = p.d_ff / p.d_model;
     split = split < 1 ? 1 : (split > 4 ? 4 : split);
     const int kb2 = p.d_ff / 64;                              // every sub-unit must own at least one K block

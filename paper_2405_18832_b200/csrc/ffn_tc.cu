@@ -56,6 +56,7 @@ constexpr int kABytes = kTileRows * 128;
 constexpr int kMaxStages = 10;
 constexpr int kQueue = 4;            // unit ids in flight between the producer and the other roles
 constexpr int kHotTokTile = 256, kHotStages = 4;     // 4 x (16 KB + 32 KB)
+constexpr int kColdTilesPerUnit = 2;  // a cold unit covers two 128-feature tiles that share one token tile
 constexpr int kTileBytes = 192 * 1024;
 constexpr int kNumBars = 2 * kMaxStages + 6 + 2 * kQueue;
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
@@ -114,7 +115,8 @@ struct Unit {
     int kb0, kb1;   // K blocks [kb0, kb1) of the reduction handled by this unit
     int split;      // sub-unit index along K, n_split - 1 = the one that finishes the tile
     int n_split;    // sub-units of this tile (1 unless cold second layer)
-    int tile_idx;   // cold second-layer tile index (partials / part_done)
+    int tile_idx;   // cold second-layer unit index (partials / part_done)
+    int tiles;      // 128-feature tiles of this unit: 1 (hot) or up to 2 (cold) sharing one token tile
 };
 
 static_assert(sizeof(Unit) <= 64, "unit queue slots are 64 bytes");
@@ -129,6 +131,7 @@ struct UnitTable {
     int* tt;          // token tiles of this expert
     int* per;         // tokens per tile (multiple of 16)
     int n_hot, n_all, nt1, nt2;      // 128-feature tiles of layer 1 (d_ff) and layer 2 (d_model)
+    int nt1c, nt2c;                  // cold units per token tile: pairs of feature tiles
     int kblocks1, kblocks2;          // 64-wide K blocks of layer 1 (d_model) and layer 2 (d_ff)
     int n_split, kb_per_split;
     int seg1, seg2, seg3, total_units;   // list = [hot L1 | hot L2 | cold L1 | cold L2 (split)]
@@ -148,7 +151,7 @@ struct UnitTable {
             r.split = v % n_split;
             v /= n_split;
         }
-        const int ntl = r.layer ? nt2 : nt1;
+        const int ntl = r.cold ? (r.layer ? nt2c : nt1c) : (r.layer ? nt2 : nt1);
         const int lo_entry = r.cold ? n_hot : 0;
         const int tt_base = tt_prefix[lo_entry];
         int lo = lo_entry, hi = (r.cold ? n_all : n_hot) - 1;      // largest entry with block start <= v
@@ -160,13 +163,14 @@ struct UnitTable {
         const int tok = local % tt[lo];
         const int ntile = local / tt[lo];
         r.e = e[lo];
-        r.n0 = ntile * kTileRows;
+        r.n0 = ntile * kTileRows * (r.cold ? kColdTilesPerUnit : 1);
+        r.tiles = r.cold ? min(kColdTilesPerUnit, (r.layer ? nt2 : nt1) - kColdTilesPerUnit * ntile) : 1;
         const int r_in_e = tok * per[lo];
         r.rows = min(per[lo], m[lo] - r_in_e);
         r.nt = (r.rows + 15) & ~15;
         r.row0 = off[lo] + r_in_e;
         r.ready_idx = tt_prefix[lo] + tok;
-        r.tile_idx = (tt_prefix[lo] - tt_base + tok) * nt2 + ntile;
+        r.tile_idx = (tt_prefix[lo] - tt_base + tok) * nt2c + ntile;
         const int kb_all = r.layer ? kblocks2 : kblocks1;
         r.kb0 = r.n_split > 1 ? r.split * kb_per_split : 0;
         r.kb1 = r.n_split > 1 ? min(kb_all, r.kb0 + kb_per_split) : kb_all;
@@ -271,6 +275,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     ut.n_all = min(ut.n_hot + P.n_hot_cold[1], kMaxExperts);
     ut.nt1 = (P.d_ff + kTileRows - 1) / kTileRows;
     ut.nt2 = (P.d_model + kTileRows - 1) / kTileRows;
+    ut.nt1c = (ut.nt1 + kColdTilesPerUnit - 1) / kColdTilesPerUnit;
+    ut.nt2c = (ut.nt2 + kColdTilesPerUnit - 1) / kColdTilesPerUnit;
     for (int i = tid; i < ut.n_all; i += kThreads) {
         const bool cold = i >= ut.n_hot;
         const int e = cold ? P.cold_ids[i - ut.n_hot] : P.hot_ids[i];
@@ -320,11 +326,10 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     ut.kb_per_split = (ut.kblocks2 + P.n_split - 1) / P.n_split;
     ut.seg1 = tt_hot * ut.nt1;
     ut.seg2 = ut.seg1 + tt_hot * ut.nt2;
-    ut.seg3 = ut.seg2 + (tt_all - tt_hot) * ut.nt1;
-    ut.total_units = ut.seg3 + (tt_all - tt_hot) * ut.nt2 * P.n_split;
+    ut.seg3 = ut.seg2 + (tt_all - tt_hot) * ut.nt1c;
+    ut.total_units = ut.seg3 + (tt_all - tt_hot) * ut.nt2c * P.n_split;
     const uint32_t tiles_u32 = smem_u32(smem);
-    const int ready_target = ut.nt1;
-    const int cold_stage_bytes = kABytes + P.cold_tile * 128;
+    const int cold_stage_bytes = kColdTilesPerUnit * kABytes + P.cold_tile * 128;
     const int hot_stage_bytes = kABytes + kHotTokTile * 128;
 
     // The producer decodes every unit once, one unit ahead of its loads, and hands the decoded
@@ -350,7 +355,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first();   // weights are read once
             const uint64_t pol_x = policy_evict_last();    // token tiles are re-read by every feature tile
-            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes;
+            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes, b_off = kABytes;
             uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
             bool ok = true;
             // Publishes unit number `j` of this CTA (or the end marker) to the other roles.
@@ -384,6 +389,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     cls = un.cold;
                     stages = cls ? P.cold_stages : kHotStages;
                     stage_bytes = cls ? cold_stage_bytes : hot_stage_bytes;
+                    b_off = cls ? kColdTilesPerUnit * kABytes : kABytes;
                     stage = 0;
                 }
                 const CUtensorMap* mw = un.layer ? &map_w2 : &map_w1;
@@ -409,11 +415,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     if (kb == un.kb0) trace_time(P, it, 1);
                     const uint32_t full = full_bar(stage);
                     const uint32_t a_dst = tiles_u32 + stage * stage_bytes;
-                    mbar_arrive_expect_tx(full, kABytes + un.nt * 128);
-                    tma_load_2d(a_dst, mw, full, kb * kBlockK, un.e * N + un.n0, pol_w);
+                    mbar_arrive_expect_tx(full, un.tiles * kABytes + un.nt * 128);
+                    for (int t = 0; t < un.tiles; ++t)
+                        tma_load_2d(a_dst + t * kABytes, mw, full, kb * kBlockK, un.e * N + un.n0 + t * kTileRows, pol_w);
                     if (kb == un.kb0 && un.layer == 1) {
                         // the hidden rows of this token tile must be complete; weights already stream
                         const int32_t* flag = P.ready + un.ready_idx;
+                        const int ready_target = un.cold ? ut.nt1c : ut.nt1;   // first-layer units per token tile
                         if (ld_acquire(flag) < ready_target) {
                             const uint64_t t0 = global_timer_ns();
                             while (ld_acquire(flag) < ready_target) {
@@ -428,7 +436,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                         fence_proxy_async_all();
                     }
                     for (int j = 0; j < un.nt; j += 16)
-                        tma_load_2d(a_dst + kABytes + j * 128, mi, full, kb * kBlockK, un.row0 + j, pol_x);
+                        tma_load_2d(a_dst + b_off + j * 128, mi, full, kb * kBlockK, un.row0 + j, pol_x);
                     fill_bits ^= 1u << stage;
                     if (++stage == stages) stage = 0;
                 }
@@ -439,7 +447,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     } else if (warp == 1) {
         // ---- MMA issuer --------------------------------------------------------------
         if (lane == 0) {
-            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes;
+            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes, b_off = kABytes;
             uint32_t use_bits = 0;      // bit s: parity of the number of uses of stage s
             bool ok = true;
             for (int it = 0; ok; ++it) {
@@ -449,6 +457,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     cls = un.cold;
                     stages = cls ? P.cold_stages : kHotStages;
                     stage_bytes = cls ? cold_stage_bytes : hot_stage_bytes;
+                    b_off = cls ? kColdTilesPerUnit * kABytes : kABytes;
                     stage = 0;
                 }
                 const int b = it & 1;
@@ -469,11 +478,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     tc_fence_after_sync();
                     if (kb == un.kb0) trace_time(P, it, 3);
                     const uint32_t a_addr = tiles_u32 + stage * stage_bytes;
-                    const uint64_t a_desc = smem_desc_sw128(a_addr);
-                    const uint64_t b_desc = smem_desc_sw128(a_addr + kABytes);
+                    const uint64_t b_desc = smem_desc_sw128(a_addr + b_off);
+                    for (int t = 0; t < un.tiles; ++t) {      // feature tiles share the token tile
+                        const uint64_t a_desc = smem_desc_sw128(a_addr + t * kABytes);
 #pragma unroll
-                    for (int k4 = 0; k4 < kBlockK / 16; ++k4)
-                        umma_bf16(d_tmem, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kb != un.kb0) | (k4 != 0));
+                        for (int k4 = 0; k4 < kBlockK / 16; ++k4)
+                            umma_bf16(d_tmem + t * 128, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kb != un.kb0) | (k4 != 0));
+                    }
                     umma_commit(empty_bar(stage));   // stage reusable once these MMAs finish
                     use_bits ^= 1u << stage;
                     if (++stage == stages) stage = 0;
@@ -507,21 +518,6 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             if (warp == 2 && lane == 0) trace_time(P, it, 5);
             const int N = un.layer ? P.d_model : P.d_ff;
             const __nv_bfloat16* bias = un.layer ? P.b2 : P.b1;
-            const int n = un.n0 + q * 32 + lane;
-            const float bias_v = (bias != nullptr && n < N) ? __bfloat162float(bias[static_cast<int64_t>(un.e) * N + n]) : 0.0f;
-            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 256;
-            __nv_bfloat16* out = un.layer ? P.y : P.h;
-            const int et = tid - 64;                    // 0..127 within the epilogue warps (warps 2-5)
-            const int rd_row = et >> 4, rd_col = (et & 15) * 8;
-            const bool col_ok = un.n0 + rd_col < N;     // N is a multiple of 64: 8-wide groups are all in or all out
-            // Each group of 16 tokens is transposed through shared memory so that global stores are
-            // 16-byte pieces of 256-byte contiguous row segments.  The code is kept small on purpose:
-            // a widely unrolled epilogue with an inlined library erf per element overflowed the
-            // instruction cache and ran 20x slower.
-            // K-split tiles: fp32 partials live as [split][token][feature] so that a warp touches
-            // 128 contiguous bytes per token.
-            float* part = P.partials + static_cast<size_t>(un.tile_idx) * (un.n_split - 1) * (P.cold_tile * kTileRows) +
-                          q * 32 + lane;
             const bool is_partial = un.split + 1 < un.n_split;
             if (un.n_split > 1 && !is_partial) {
                 // finishing sub-unit: the partial tiles were taken from the list before this one
@@ -537,6 +533,25 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                 }
                 __syncwarp();
             }
+            int grp = 0;       // running 16-token group count: alternates the two staging buffers
+#pragma unroll 1
+            for (int ft = 0; ft < un.tiles; ++ft) {
+            const int n0 = un.n0 + ft * kTileRows;
+            const int n = n0 + q * 32 + lane;
+            const float bias_v = (bias != nullptr && n < N) ? __bfloat162float(bias[static_cast<int64_t>(un.e) * N + n]) : 0.0f;
+            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 256 + ft * 128;
+            __nv_bfloat16* out = un.layer ? P.y : P.h;
+            const int et = tid - 64;                    // 0..127 within the epilogue warps (warps 2-5)
+            const int rd_row = et >> 4, rd_col = (et & 15) * 8;
+            const bool col_ok = n0 + rd_col < N;     // N is a multiple of 64: 8-wide groups are all in or all out
+            // Each group of 16 tokens is transposed through shared memory so that global stores are
+            // 16-byte pieces of 256-byte contiguous row segments.  The code is kept small on purpose:
+            // a widely unrolled epilogue with an inlined library erf per element overflowed the
+            // instruction cache and ran 20x slower.
+            // K-split tiles: fp32 partials live as [split][token][feature] so that a warp touches
+            // 128 contiguous bytes per token.
+            float* part = P.partials + static_cast<size_t>(un.tile_idx * kColdTilesPerUnit + ft) * (un.n_split - 1) *
+                                           (P.cold_tile * kTileRows) + q * 32 + lane;
             // One group = 16 tokens.  mode: 0 first layer (activation), 1 second layer, 2 second
             // layer finishing a K-split tile (adds the partial tiles), 3 partial tile (fp32 store).
             const int mode = un.layer == 0 ? 0 : (un.n_split == 1 ? 1 : (is_partial ? 3 : 2));
@@ -547,7 +562,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                         part[(un.split * P.cold_tile + c0 + j) * kTileRows] = __uint_as_float(v[j]);
                     return;
                 }
-                __nv_bfloat16* sb = stg + ((c0 >> 4) & 1) * (16 * kTileRows) + q * 32 + lane;
+                __nv_bfloat16* sb = stg + (grp & 1) * (16 * kTileRows) + q * 32 + lane;
                 if (mode == 0) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
@@ -571,13 +586,14 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                         sb[j * kTileRows] = __float2bfloat16_rn(acc[j] + __uint_as_float(v[j]) + bias_v);
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                const __nv_bfloat16* rb = stg + ((c0 >> 4) & 1) * (16 * kTileRows);
+                const __nv_bfloat16* rb = stg + (grp & 1) * (16 * kTileRows);
+                ++grp;
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     const int r = rd_row + half * 8;
                     if (col_ok && c0 + r < un.rows) {
                         const uint4 val = *reinterpret_cast<const uint4*>(rb + r * kTileRows + rd_col);
-                        *reinterpret_cast<uint4*>(out + static_cast<int64_t>(un.row0 + c0 + r) * N + un.n0 + rd_col) = val;
+                        *reinterpret_cast<uint4*>(out + static_cast<int64_t>(un.row0 + c0 + r) * N + n0 + rd_col) = val;
                     }
                 }
             };
@@ -596,6 +612,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     drain16(vb, c0 + 16);
                 }
             }
+            }   // feature tiles of the unit
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
@@ -647,7 +664,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         if (last) {
             for (int i = lane; i < tt_all; i += 32) P.ready[i] = 0;
             if (P.n_split > 1)
-                for (int i = lane; i < (tt_all - tt_hot) * ut.nt2; i += 32) P.part_done[i] = 0;
+                for (int i = lane; i < (tt_all - tt_hot) * ut.nt2c; i += 32) P.part_done[i] = 0;
             if (lane == 0) {
                 *P.next_unit = 0;
                 *P.ticket = 0;
@@ -733,7 +750,7 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.ticket = reinterpret_cast<int32_t*>(base + WsLayout::kCounters);
     P.next_unit = P.ticket + 1;
     P.cold_tile = cold_token_tile(p);
-    P.cold_stages = std::min(kMaxStages, kTileBytes / (kABytes + P.cold_tile * 128));
+    P.cold_stages = std::min(kMaxStages, kTileBytes / (kColdTilesPerUnit * kABytes + P.cold_tile * 128));
     const WsLayout L = ws_layout(p);
     P.n_split = L.n_split;
     P.part_done = reinterpret_cast<int32_t*>(base + L.part_done_off);
