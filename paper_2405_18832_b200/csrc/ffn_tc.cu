@@ -12,10 +12,17 @@
 // output features of the expert's weight matrix and the MMA N dimension holds the tokens,
 // so an expert with m tokens costs one pass over its weights with N = m rounded up to 16.
 // The class chosen by the router selects the tiling of a work unit:
-//   hot : token tile <= 256 (a full-rate 128 x 256 MMA), 4-stage ring of 48 KB stages;
-//   cold: token tile = threshold-1 rounded up to 16 (at most 64), 8 to 10 stages of 18-24 KB
-//         -> a deep queue of weight bytes in flight per SM; the tensor core idles most of
-//         the time and HBM sets the pace.
+// A unit covers two 128-feature tiles that share one token tile (the token tile is the
+// operand that every feature tile re-reads through L2, so pairing halves that traffic).
+//   hot : token tile <= 256 (full-rate 128 x 256 MMAs).  For d_model >= 1536 a unit
+//         takes two feature tiles: 3 stages of 64 KB, and the two accumulators fill all 512
+//         TMEM columns, so the epilogue is not overlapped with the next unit's MMAs - cheaper
+//         than re-reading a 32 KB token tile per 16 KB weight tile.  For smaller layers the
+//         exposed epilogue and the halved unit count cost more than they save: one feature
+//         tile per unit, 4 stages of 48 KB, two accumulator buffers;
+//   cold: token tile = threshold-1 rounded up to 16 (at most 64), 4 or 5 stages of 34-40 KB,
+//         two accumulator buffers -> a deep queue of weight bytes in flight per SM; the tensor
+//         core idles most of the time and HBM sets the pace.
 // Work units (expert, 128-feature tile, token tile) form one ordered list: hot first
 // layer, hot second layer, cold first layer, cold second layer.  One persistent CTA per SM
 // takes the next unit from a device-wide counter.  A second-layer unit needs the hidden
@@ -55,8 +62,8 @@ constexpr int kTileRows = 128;        // output features per unit = MMA M
 constexpr int kABytes = kTileRows * 128;
 constexpr int kMaxStages = 10;
 constexpr int kQueue = 4;            // unit ids in flight between the producer and the other roles
-constexpr int kHotTokTile = 256, kHotStages = 4;     // 4 x (16 KB + 32 KB)
-constexpr int kColdTilesPerUnit = 2;  // a cold unit covers two 128-feature tiles that share one token tile
+constexpr int kHotTokTile = 256;
+constexpr int kTilesPerUnit = 2;      // a unit covers two 128-feature tiles that share one token tile
 constexpr int kTileBytes = 192 * 1024;
 constexpr int kNumBars = 2 * kMaxStages + 6 + 2 * kQueue;
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
@@ -70,7 +77,8 @@ enum WaitSite { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3,
 
 struct FfnParams {
     int d_model, d_ff, act;
-    int cold_tile, cold_stages;   // stage geometry of the cold class
+    int cold_tile;                // token tile of the cold class
+    int pair_mask;                // bit (class * 2 + layer): units of that segment take two feature tiles
     int n_split;                  // K-splits of a cold second-layer unit (1 = none)
     const __nv_bfloat16* b1;
     const __nv_bfloat16* b2;
@@ -116,7 +124,8 @@ struct Unit {
     int split;      // sub-unit index along K, n_split - 1 = the one that finishes the tile
     int n_split;    // sub-units of this tile (1 unless cold second layer)
     int tile_idx;   // cold second-layer unit index (partials / part_done)
-    int tiles;      // 128-feature tiles of this unit: 1 (hot) or up to 2 (cold) sharing one token tile
+    int tiles;      // 128-feature tiles of this unit (1 or 2) sharing one token tile
+    int wide;       // 1: the unit's accumulators occupy all 512 TMEM columns (hot, two tiles)
 };
 
 static_assert(sizeof(Unit) <= 64, "unit queue slots are 64 bytes");
@@ -131,7 +140,8 @@ struct UnitTable {
     int* tt;          // token tiles of this expert
     int* per;         // tokens per tile (multiple of 16)
     int n_hot, n_all, nt1, nt2;      // 128-feature tiles of layer 1 (d_ff) and layer 2 (d_model)
-    int nt1c, nt2c;                  // cold units per token tile: pairs of feature tiles
+    int upt[4];                      // units per token tile, by segment (class * 2 + layer)
+    int tpu[4];                      // feature tiles per unit, by segment
     int kblocks1, kblocks2;          // 64-wide K blocks of layer 1 (d_model) and layer 2 (d_ff)
     int n_split, kb_per_split;
     int seg1, seg2, seg3, total_units;   // list = [hot L1 | hot L2 | cold L1 | cold L2 (split)]
@@ -151,7 +161,8 @@ struct UnitTable {
             r.split = v % n_split;
             v /= n_split;
         }
-        const int ntl = r.cold ? (r.layer ? nt2c : nt1c) : (r.layer ? nt2 : nt1);
+        const int sgm = r.cold * 2 + r.layer;
+        const int ntl = upt[sgm];
         const int lo_entry = r.cold ? n_hot : 0;
         const int tt_base = tt_prefix[lo_entry];
         int lo = lo_entry, hi = (r.cold ? n_all : n_hot) - 1;      // largest entry with block start <= v
@@ -163,14 +174,15 @@ struct UnitTable {
         const int tok = local % tt[lo];
         const int ntile = local / tt[lo];
         r.e = e[lo];
-        r.n0 = ntile * kTileRows * (r.cold ? kColdTilesPerUnit : 1);
-        r.tiles = r.cold ? min(kColdTilesPerUnit, (r.layer ? nt2 : nt1) - kColdTilesPerUnit * ntile) : 1;
+        r.n0 = ntile * kTileRows * tpu[sgm];
+        r.tiles = min(tpu[sgm], (r.layer ? nt2 : nt1) - tpu[sgm] * ntile);
+        r.wide = !r.cold && tpu[sgm] == 2;
         const int r_in_e = tok * per[lo];
         r.rows = min(per[lo], m[lo] - r_in_e);
         r.nt = (r.rows + 15) & ~15;
         r.row0 = off[lo] + r_in_e;
         r.ready_idx = tt_prefix[lo] + tok;
-        r.tile_idx = (tt_prefix[lo] - tt_base + tok) * nt2c + ntile;
+        r.tile_idx = (tt_prefix[lo] - tt_base + tok) * upt[3] + ntile;
         const int kb_all = r.layer ? kblocks2 : kblocks1;
         r.kb0 = r.n_split > 1 ? r.split * kb_per_split : 0;
         r.kb1 = r.n_split > 1 ? min(kb_all, r.kb0 + kb_per_split) : kb_all;
@@ -275,8 +287,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     ut.n_all = min(ut.n_hot + P.n_hot_cold[1], kMaxExperts);
     ut.nt1 = (P.d_ff + kTileRows - 1) / kTileRows;
     ut.nt2 = (P.d_model + kTileRows - 1) / kTileRows;
-    ut.nt1c = (ut.nt1 + kColdTilesPerUnit - 1) / kColdTilesPerUnit;
-    ut.nt2c = (ut.nt2 + kColdTilesPerUnit - 1) / kColdTilesPerUnit;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        ut.tpu[g] = ((P.pair_mask >> g) & 1) + 1;
+        ut.upt[g] = (((g & 1) ? ut.nt2 : ut.nt1) + ut.tpu[g] - 1) / ut.tpu[g];
+    }
     for (int i = tid; i < ut.n_all; i += kThreads) {
         const bool cold = i >= ut.n_hot;
         const int e = cold ? P.cold_ids[i - ut.n_hot] : P.hot_ids[i];
@@ -324,13 +339,15 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     ut.kblocks2 = P.d_ff / kBlockK;
     ut.n_split = P.n_split;
     ut.kb_per_split = (ut.kblocks2 + P.n_split - 1) / P.n_split;
-    ut.seg1 = tt_hot * ut.nt1;
-    ut.seg2 = ut.seg1 + tt_hot * ut.nt2;
-    ut.seg3 = ut.seg2 + (tt_all - tt_hot) * ut.nt1c;
-    ut.total_units = ut.seg3 + (tt_all - tt_hot) * ut.nt2c * P.n_split;
+    ut.seg1 = tt_hot * ut.upt[0];
+    ut.seg2 = ut.seg1 + tt_hot * ut.upt[1];
+    ut.seg3 = ut.seg2 + (tt_all - tt_hot) * ut.upt[2];
+    ut.total_units = ut.seg3 + (tt_all - tt_hot) * ut.upt[3] * P.n_split;
     const uint32_t tiles_u32 = smem_u32(smem);
-    const int cold_stage_bytes = kColdTilesPerUnit * kABytes + P.cold_tile * 128;
-    const int hot_stage_bytes = kABytes + kHotTokTile * 128;
+    // Stage geometry of a segment: its weight tiles, then the token tile; as many stages as fit.
+    auto geom_b_off = [&](int g) { return ut.tpu[g] * kABytes; };
+    auto geom_stage_bytes = [&](int g) { return ut.tpu[g] * kABytes + ((g & 2) ? P.cold_tile : kHotTokTile) * 128; };
+    auto geom_stages = [&](int g) { return min(kMaxStages, kTileBytes / geom_stage_bytes(g)); };
 
     // The producer decodes every unit once, one unit ahead of its loads, and hands the decoded
     // record to the other roles through a small shared-memory queue (decoding costs about half
@@ -350,12 +367,34 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         return un;
     };
 
+    // Accumulator buffers.  A narrow unit (cold, or hot with one feature tile) uses one of two
+    // 256-column buffers in turn (its tiles at +0 and +128); a wide unit (hot, two tiles of up
+    // to 256 tokens) fills all 512 columns (tiles at 0 and 256) and is tracked as buffer 0.
+    // The narrow unit that follows a wide one starts again at buffer 0, so waiting for that
+    // buffer also waits for the wide unit's drain; a wide unit that follows narrow ones
+    // additionally waits for buffer 1 (see the MMA issuer).  Every role walks the same
+    // sequence and keeps the same counts.
+    struct AccCursor {
+        int uses0 = 0, uses1 = 0;
+        int seq = 0;
+        int b = 0;
+        uint32_t parity = 0;        // parity of this use of buffer b (full: wait parity, empty: wait parity ^ 1)
+        uint32_t other_parity = 0;  // parity that tells buffer 1's latest use has been drained (wide units)
+        __device__ void next(const Unit& un) {
+            b = un.wide ? 0 : (seq++ & 1);
+            if (un.wide) seq = 0;
+            other_parity = (uses1 & 1) ^ 1;
+            if (b == 0) { parity = uses0 & 1; ++uses0; } else { parity = uses1 & 1; ++uses1; }
+        }
+    };
+    auto acc_col = [](const Unit& un, int b, int t) { return un.wide ? t * 256 : b * 256 + t * 128; };
+
     if (warp == 0) {
         // ---- scheduler + TMA producer ------------------------------------------------------
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first();   // weights are read once
             const uint64_t pol_x = policy_evict_last();    // token tiles are re-read by every feature tile
-            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes, b_off = kABytes;
+            int stage = 0, cls = -1, stages = 1, stage_bytes = 0, b_off = 0;
             uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
             bool ok = true;
             // Publishes unit number `j` of this CTA (or the end marker) to the other roles.
@@ -378,18 +417,20 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             for (int it = 0; ok && cur.id >= 0; ++it) {
                 const Unit un = cur;
                 trace_mark(P, it, 0, static_cast<unsigned long long>(un.id));
-                if (un.cold != cls) {
+                if (un.cold * 2 + un.layer != cls &&
+                    (cls < 0 || geom_stage_bytes(un.cold * 2 + un.layer) != stage_bytes ||
+                     geom_b_off(un.cold * 2 + un.layer) != b_off)) {
                     // geometry switch: every stage filled so far must have been consumed
-                    for (int s = 0; ok && s < stages; ++s)
+                    for (int s = 0; ok && cls >= 0 && s < stages; ++s)
                         if (!mbar_wait(empty_bar(s), ((fill_bits >> s) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                             report_timeout(P.status, abort_flag, kSiteDrain);
                             ok = false;
                         }
                     if (!ok) break;
-                    cls = un.cold;
-                    stages = cls ? P.cold_stages : kHotStages;
-                    stage_bytes = cls ? cold_stage_bytes : hot_stage_bytes;
-                    b_off = cls ? kColdTilesPerUnit * kABytes : kABytes;
+                    cls = un.cold * 2 + un.layer;
+                    stages = geom_stages(cls);
+                    stage_bytes = geom_stage_bytes(cls);
+                    b_off = geom_b_off(cls);
                     stage = 0;
                 }
                 const CUtensorMap* mw = un.layer ? &map_w2 : &map_w1;
@@ -421,7 +462,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                     if (kb == un.kb0 && un.layer == 1) {
                         // the hidden rows of this token tile must be complete; weights already stream
                         const int32_t* flag = P.ready + un.ready_idx;
-                        const int ready_target = un.cold ? ut.nt1c : ut.nt1;   // first-layer units per token tile
+                        const int ready_target = ut.upt[un.cold * 2];   // first-layer units per token tile
                         if (ld_acquire(flag) < ready_target) {
                             const uint64_t t0 = global_timer_ns();
                             while (ld_acquire(flag) < ready_target) {
@@ -447,28 +488,31 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     } else if (warp == 1) {
         // ---- MMA issuer --------------------------------------------------------------
         if (lane == 0) {
-            int stage = 0, cls = -1, stages = kHotStages, stage_bytes = hot_stage_bytes, b_off = kABytes;
+            int stage = 0, cls = -1, stages = 1, stage_bytes = 0, b_off = 0;
             uint32_t use_bits = 0;      // bit s: parity of the number of uses of stage s
             bool ok = true;
+            AccCursor acc;
             for (int it = 0; ok; ++it) {
                 const Unit un = pop_unit(it, false);
                 if (un.id < 0) break;
-                if (un.cold != cls) {
-                    cls = un.cold;
-                    stages = cls ? P.cold_stages : kHotStages;
-                    stage_bytes = cls ? cold_stage_bytes : hot_stage_bytes;
-                    b_off = cls ? kColdTilesPerUnit * kABytes : kABytes;
+                if (un.cold * 2 + un.layer != cls &&
+                    (cls < 0 || geom_stage_bytes(un.cold * 2 + un.layer) != stage_bytes ||
+                     geom_b_off(un.cold * 2 + un.layer) != b_off)) {
+                    cls = un.cold * 2 + un.layer;
+                    stages = geom_stages(cls);
+                    stage_bytes = geom_stage_bytes(cls);
+                    b_off = geom_b_off(cls);
                     stage = 0;
                 }
-                const int b = it & 1;
-                const uint32_t tphase = (it >> 1) & 1;
-                if (!mbar_wait(acc_empty(b), tphase ^ 1u, abort_flag, kWaitLimitNs)) {
+                acc.next(un);
+                const int b = acc.b;
+                if (!mbar_wait(acc_empty(b), acc.parity ^ 1u, abort_flag, kWaitLimitNs) ||
+                    (un.wide && !mbar_wait(acc_empty(1), acc.other_parity, abort_flag, kWaitLimitNs))) {
                     report_timeout(P.status, abort_flag, kSiteMmaTmemEmpty);
                     break;
                 }
                 tc_fence_after_sync();
                 const uint32_t idesc = idesc_bf16_m128(un.nt);
-                const uint32_t d_tmem = tmem_base + b * 256;
                 for (int kb = un.kb0; kb < un.kb1; ++kb) {
                     if (!mbar_wait(full_bar(stage), (use_bits >> stage) & 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteMmaFull);
@@ -483,7 +527,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                         const uint64_t a_desc = smem_desc_sw128(a_addr + t * kABytes);
 #pragma unroll
                         for (int k4 = 0; k4 < kBlockK / 16; ++k4)
-                            umma_bf16(d_tmem + t * 128, a_desc + 2 * k4, b_desc + 2 * k4, idesc, (kb != un.kb0) | (k4 != 0));
+                            umma_bf16(tmem_base + acc_col(un, b, t), a_desc + 2 * k4, b_desc + 2 * k4, idesc,
+                                      (kb != un.kb0) | (k4 != 0));
                     }
                     umma_commit(empty_bar(stage));   // stage reusable once these MMAs finish
                     use_bits ^= 1u << stage;
@@ -496,13 +541,14 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     } else if (warp < 6) {
         // ---- epilogue: TMEM -> registers -> bias, activation -> shared -> global -------------
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        AccCursor acc;
         for (int it = 0;; ++it) {
             const Unit un = pop_unit(it, true);
-            const int b = it & 1;
-            const uint32_t tphase = (it >> 1) & 1;
             bool got = un.id >= 0;
+            if (got) acc.next(un);
+            const int b = acc.b;
             if (got) {
-                got = mbar_wait(acc_full(b), tphase, abort_flag, kWaitLimitNs);
+                got = mbar_wait(acc_full(b), acc.parity, abort_flag, kWaitLimitNs);
                 if (!got) report_timeout(P.status, abort_flag, kSiteEpilogueTmemFull);
             }
             // the four epilogue warps share a named barrier below: leave together or not at all
@@ -539,7 +585,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             const int n0 = un.n0 + ft * kTileRows;
             const int n = n0 + q * 32 + lane;
             const float bias_v = (bias != nullptr && n < N) ? __bfloat162float(bias[static_cast<int64_t>(un.e) * N + n]) : 0.0f;
-            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 256 + ft * 128;
+            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc_col(un, b, ft);
             __nv_bfloat16* out = un.layer ? P.y : P.h;
             const int et = tid - 64;                    // 0..127 within the epilogue warps (warps 2-5)
             const int rd_row = et >> 4, rd_col = (et & 15) * 8;
@@ -550,7 +596,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             // instruction cache and ran 20x slower.
             // K-split tiles: fp32 partials live as [split][token][feature] so that a warp touches
             // 128 contiguous bytes per token.
-            float* part = P.partials + static_cast<size_t>(un.tile_idx * kColdTilesPerUnit + ft) * (un.n_split - 1) *
+            float* part = P.partials + static_cast<size_t>(un.tile_idx * kTilesPerUnit + ft) * (un.n_split - 1) *
                                            (P.cold_tile * kTileRows) + q * 32 + lane;
             // One group = 16 tokens.  mode: 0 first layer (activation), 1 second layer, 2 second
             // layer finishing a K-split tile (adds the partial tiles), 3 partial tile (fp32 store).
@@ -628,11 +674,12 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         // that wait off the epilogue warps.  Order: epilogue stores -> mbarrier (release/acquire
         // at CTA scope) -> this thread's device-scope fence (cumulative) -> counter increment.
         if (lane == 0) {
+            AccCursor acc;
             for (int it = 0;; ++it) {
                 const Unit un = pop_unit(it, false);
                 if (un.id < 0) break;
-                const int b = it & 1;
-                if (!mbar_wait(rows_stored(b), (it >> 1) & 1, abort_flag, kWaitLimitNs))
+                acc.next(un);
+                if (!mbar_wait(rows_stored(acc.b), acc.parity, abort_flag, kWaitLimitNs))
                     break;   // the role that stalled has already reported
                 if (un.layer == 0) {
                     __threadfence();
@@ -664,7 +711,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         if (last) {
             for (int i = lane; i < tt_all; i += 32) P.ready[i] = 0;
             if (P.n_split > 1)
-                for (int i = lane; i < (tt_all - tt_hot) * ut.nt2c; i += 32) P.part_done[i] = 0;
+                for (int i = lane; i < (tt_all - tt_hot) * ut.upt[3]; i += 32) P.part_done[i] = 0;
             if (lane == 0) {
                 *P.next_unit = 0;
                 *P.ticket = 0;
@@ -750,7 +797,12 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.ticket = reinterpret_cast<int32_t*>(base + WsLayout::kCounters);
     P.next_unit = P.ticket + 1;
     P.cold_tile = cold_token_tile(p);
-    P.cold_stages = std::min(kMaxStages, kTileBytes / (kColdTilesPerUnit * kABytes + P.cold_tile * 128));
+    // Cold units always pair feature tiles.  Hot units pair them when d_model >= 1536: the K loop of
+    // the first layer is then long enough to pay for the exposed epilogue, and the second layer
+    // has enough feature tiles left to keep every SM busy with half as many, twice as long units
+    // (measured: pairing the hot class takes NLLB-sized layers from 1.53 to 1.39 ms and
+    // Switch-Base-sized ones from 175 to 195 us).
+    P.pair_mask = 0xC | (p.d_model >= 1536 ? 0x3 : 0);
     const WsLayout L = ws_layout(p);
     P.n_split = L.n_split;
     P.part_done = reinterpret_cast<int32_t*>(base + L.part_done_off);
