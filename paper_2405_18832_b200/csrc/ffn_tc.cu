@@ -56,16 +56,17 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 224;       // producer, MMA, 4 epilogue warps, publisher
+constexpr int kThreads = 256;       // weight producer, MMA, 4 epilogue warps, publisher, token-tile producer
 constexpr int kBlockK = 64;           // K elements per stage: one 128-byte swizzle row
 constexpr int kTileRows = 128;        // output features per unit = MMA M
 constexpr int kABytes = kTileRows * 128;
-constexpr int kMaxStages = 10;
+constexpr int kMaxStagesA = 10;       // weight-tile ring
+constexpr int kMaxStagesB = 4;        // token-tile ring
 constexpr int kQueue = 4;            // unit ids in flight between the producer and the other roles
 constexpr int kHotTokTile = 256;
 constexpr int kTilesPerUnit = 2;      // a unit covers two 128-feature tiles that share one token tile
 constexpr int kTileBytes = 192 * 1024;
-constexpr int kNumBars = 2 * kMaxStages + 6 + 2 * kQueue;
+constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue;
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
 constexpr int kStageOutBytes = 2 * 16 * kTileRows * 2;
 constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kQueue * 64 + kTableInts * 4 + kStageOutBytes + 16;
@@ -220,10 +221,18 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
+// Tensor maps, all 64 columns (128 bytes) wide with the 128-byte swizzle.  Weights: boxes of 128
+// and 256 rows (one or two feature tiles per copy).  Token rows (x_perm for layer 1, hidden
+// activations for layer 2): boxes of 16, 64 and 256 rows, so that a token tile of any multiple
+// of 16 rows is covered by a few large copies (sixteen 2 KB copies per 32 KB token tile made
+// the TMA issue rate, not bandwidth, the limit of the hot class).
+struct FfnMaps {
+    CUtensorMap w[2][2];      // [layer][0: 128 rows, 1: 256 rows]
+    CUtensorMap in[2][3];     // [layer][0: 16 rows, 1: 64 rows, 2: 256 rows]
+};
+
 template <int kAct>
-__global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
-        const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
-        const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_h, const FfnParams P) {
+__global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_constant__ FfnMaps M, const FfnParams P) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kTileBytes);
@@ -243,13 +252,16 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
 
     // barrier addresses
     const uint32_t bar0 = smem_u32(bars);
-    auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
-    auto acc_full = [&](int b) { return bar0 + 8u * (2 * kMaxStages + b); };
-    auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 2 + b); };
-    auto rows_stored = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 4 + b); };
-    auto q_full = [&](int s) { return bar0 + 8u * (2 * kMaxStages + 6 + s); };
-    auto q_empty = [&](int s) { return bar0 + 8u * (2 * kMaxStages + 6 + kQueue + s); };
+    constexpr int kRingBars = 2 * kMaxStagesA + 2 * kMaxStagesB;
+    auto full_a = [&](int s) { return bar0 + 8u * s; };
+    auto empty_a = [&](int s) { return bar0 + 8u * (kMaxStagesA + s); };
+    auto full_b = [&](int s) { return bar0 + 8u * (2 * kMaxStagesA + s); };
+    auto empty_b = [&](int s) { return bar0 + 8u * (2 * kMaxStagesA + kMaxStagesB + s); };
+    auto acc_full = [&](int b) { return bar0 + 8u * (kRingBars + b); };
+    auto acc_empty = [&](int b) { return bar0 + 8u * (kRingBars + 2 + b); };
+    auto rows_stored = [&](int b) { return bar0 + 8u * (kRingBars + 4 + b); };
+    auto q_full = [&](int s) { return bar0 + 8u * (kRingBars + 6 + s); };
+    auto q_empty = [&](int s) { return bar0 + 8u * (kRingBars + 6 + kQueue + s); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -258,9 +270,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     pdl_launch_dependents();
     if (tid == 0) {
         *abort_flag = 0;
-        for (int s = 0; s < kMaxStages; ++s) {
-            mbar_init(full_bar(s), 1);    // producer's expect_tx arrival
-            mbar_init(empty_bar(s), 1);   // one tcgen05.commit
+        for (int s = 0; s < kMaxStagesA; ++s) {
+            mbar_init(full_a(s), 1);    // weight producer's expect_tx arrival
+            mbar_init(empty_a(s), 1);   // one tcgen05.commit
+        }
+        for (int s = 0; s < kMaxStagesB; ++s) {
+            mbar_init(full_b(s), 1);    // token-tile producer's expect_tx arrival
+            mbar_init(empty_b(s), 1);   // one tcgen05.commit
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full(b), 1);      // one commit
@@ -269,13 +285,14 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         }
         for (int s = 0; s < kQueue; ++s) {
             mbar_init(q_full(s), 1);        // producer
-            mbar_init(q_empty(s), 6);       // MMA issuer, 4 epilogue warps, publisher
+            mbar_init(q_empty(s), 7);       // MMA issuer, 4 epilogue warps, publisher, token-tile producer
         }
         fence_barrier_init();
-        prefetch_tensormap(&map_w1);
-        prefetch_tensormap(&map_w2);
-        prefetch_tensormap(&map_x);
-        prefetch_tensormap(&map_h);
+        for (int l = 0; l < 2; ++l) {
+            prefetch_tensormap(&M.w[l][0]);
+            prefetch_tensormap(&M.w[l][1]);
+            for (int i = 0; i < 3; ++i) prefetch_tensormap(&M.in[l][i]);
+        }
     } else if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), kTmemCols);
         tmem_relinquish();
@@ -344,10 +361,24 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
     ut.seg3 = ut.seg2 + (tt_all - tt_hot) * ut.upt[2];
     ut.total_units = ut.seg3 + (tt_all - tt_hot) * ut.upt[3] * P.n_split;
     const uint32_t tiles_u32 = smem_u32(smem);
-    // Stage geometry of a segment: its weight tiles, then the token tile; as many stages as fit.
-    auto geom_b_off = [&](int g) { return ut.tpu[g] * kABytes; };
-    auto geom_stage_bytes = [&](int g) { return ut.tpu[g] * kABytes + ((g & 2) ? P.cold_tile : kHotTokTile) * 128; };
-    auto geom_stages = [&](int g) { return min(kMaxStages, kTileBytes / geom_stage_bytes(g)); };
+    // Ring geometry of a segment.  Weight tiles come from DRAM (long latency) and token tiles from
+    // L2 (short latency, re-read by every feature tile), so they get separate rings: a few
+    // token-tile stages fetched just in time, and all remaining shared memory as weight stages
+    // in flight.  (With one combined ring the hot class had 48 KB of weights in flight per SM
+    // and ran at the latency limit, 77 GB/s of fill per SM.)
+    struct Geom { int a_bytes, b_bytes, na, nb, b_base; };
+    auto geom_of = [&](int g) {
+        Geom r;
+        r.a_bytes = ut.tpu[g] * kABytes;
+        r.b_bytes = ((g & 2) ? P.cold_tile : kHotTokTile) * 128;
+        r.nb = (g & 2) ? kMaxStagesB : 3;
+        r.na = min(kMaxStagesA, (kTileBytes - r.nb * r.b_bytes) / r.a_bytes);
+        r.b_base = r.na * r.a_bytes;
+        return r;
+    };
+    auto same_geom = [](const Geom& x, const Geom& y) {
+        return x.a_bytes == y.a_bytes && x.b_bytes == y.b_bytes && x.na == y.na && x.nb == y.nb;
+    };
 
     // The producer decodes every unit once, one unit ahead of its loads, and hands the decoded
     // record to the other roles through a small shared-memory queue (decoding costs about half
@@ -393,8 +424,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
         // ---- scheduler + TMA producer ------------------------------------------------------
         if (lane == 0) {
             const uint64_t pol_w = policy_evict_first();   // weights are read once
-            const uint64_t pol_x = policy_evict_last();    // token tiles are re-read by every feature tile
-            int stage = 0, cls = -1, stages = 1, stage_bytes = 0, b_off = 0;
+            int stage = 0, cls = -1;
+            Geom gm = {};
             uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
             bool ok = true;
             // Publishes unit number `j` of this CTA (or the end marker) to the other roles.
@@ -417,24 +448,22 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
             for (int it = 0; ok && cur.id >= 0; ++it) {
                 const Unit un = cur;
                 trace_mark(P, it, 0, static_cast<unsigned long long>(un.id));
-                if (un.cold * 2 + un.layer != cls &&
-                    (cls < 0 || geom_stage_bytes(un.cold * 2 + un.layer) != stage_bytes ||
-                     geom_b_off(un.cold * 2 + un.layer) != b_off)) {
-                    // geometry switch: every stage filled so far must have been consumed
-                    for (int s = 0; ok && cls >= 0 && s < stages; ++s)
-                        if (!mbar_wait(empty_bar(s), ((fill_bits >> s) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
-                            report_timeout(P.status, abort_flag, kSiteDrain);
-                            ok = false;
-                        }
-                    if (!ok) break;
+                if (un.cold * 2 + un.layer != cls) {
+                    const Geom g2 = geom_of(un.cold * 2 + un.layer);
+                    if (cls < 0 || !same_geom(g2, gm)) {
+                        // geometry switch: every stage filled so far must have been consumed
+                        for (int s = 0; ok && cls >= 0 && s < gm.na; ++s)
+                            if (!mbar_wait(empty_a(s), ((fill_bits >> s) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
+                                report_timeout(P.status, abort_flag, kSiteDrain);
+                                ok = false;
+                            }
+                        if (!ok) break;
+                        gm = g2;
+                        stage = 0;
+                    }
                     cls = un.cold * 2 + un.layer;
-                    stages = geom_stages(cls);
-                    stage_bytes = geom_stage_bytes(cls);
-                    b_off = geom_b_off(cls);
-                    stage = 0;
                 }
-                const CUtensorMap* mw = un.layer ? &map_w2 : &map_w1;
-                const CUtensorMap* mi = un.layer ? &map_h : &map_x;
+                const CUtensorMap* mw = &M.w[un.layer][un.tiles - 1];   // both feature tiles in one copy
                 const int N = un.layer ? P.d_model : P.d_ff;
                 bool next_ready = false;
                 for (int kb = un.kb0; kb < un.kb1; ++kb) {
@@ -448,61 +477,106 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                         if (!push_unit(it + 1, nxt)) { ok = false; break; }
                         next_ready = true;
                     }
-                    if (!mbar_wait(empty_bar(stage), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
+                    if (!mbar_wait(empty_a(stage), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteProducerEmpty);
                         ok = false;
                         break;
                     }
                     if (kb == un.kb0) trace_time(P, it, 1);
-                    const uint32_t full = full_bar(stage);
-                    const uint32_t a_dst = tiles_u32 + stage * stage_bytes;
-                    mbar_arrive_expect_tx(full, un.tiles * kABytes + un.nt * 128);
-                    for (int t = 0; t < un.tiles; ++t)
-                        tma_load_2d(a_dst + t * kABytes, mw, full, kb * kBlockK, un.e * N + un.n0 + t * kTileRows, pol_w);
-                    if (kb == un.kb0 && un.layer == 1) {
-                        // the hidden rows of this token tile must be complete; weights already stream
-                        const int32_t* flag = P.ready + un.ready_idx;
-                        const int ready_target = ut.upt[un.cold * 2];   // first-layer units per token tile
-                        if (ld_acquire(flag) < ready_target) {
-                            const uint64_t t0 = global_timer_ns();
-                            while (ld_acquire(flag) < ready_target) {
-                                if (*abort_flag != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
-                                    report_timeout(P.status, abort_flag, kSiteHiddenReady);
-                                    ok = false;
-                                    break;
-                                }
-                            }
-                            if (!ok) break;
-                        }
-                        fence_proxy_async_all();
-                    }
-                    for (int j = 0; j < un.nt; j += 16)
-                        tma_load_2d(a_dst + b_off + j * 128, mi, full, kb * kBlockK, un.row0 + j, pol_x);
+                    const uint32_t full = full_a(stage);
+                    const uint32_t a_dst = tiles_u32 + stage * gm.a_bytes;
+                    mbar_arrive_expect_tx(full, un.tiles * kABytes);
+                    tma_load_2d(a_dst, mw, full, kb * kBlockK, un.e * N + un.n0, pol_w);
                     fill_bits ^= 1u << stage;
-                    if (++stage == stages) stage = 0;
+                    if (++stage == gm.na) stage = 0;
                 }
                 trace_time(P, it, 2);
                 cur = nxt;
             }
         }
+    } else if (warp == 7) {
+        // ---- token-tile producer (operand B: rows of x_perm or of the hidden activations) -------
+        if (lane == 0) {
+            const uint64_t pol_x = policy_evict_last();    // token tiles are re-read by every feature tile
+            int stage = 0, cls = -1;
+            Geom gm = {};
+            uint32_t fill_bits = 0;
+            bool ok = true;
+            for (int it = 0; ok; ++it) {
+                const Unit un = pop_unit(it, false);
+                if (un.id < 0) break;
+                if (un.cold * 2 + un.layer != cls) {
+                    const Geom g2 = geom_of(un.cold * 2 + un.layer);
+                    if (cls < 0 || !same_geom(g2, gm)) {
+                        for (int s = 0; ok && cls >= 0 && s < gm.nb; ++s)
+                            if (!mbar_wait(empty_b(s), ((fill_bits >> s) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
+                                report_timeout(P.status, abort_flag, kSiteDrain);
+                                ok = false;
+                            }
+                        if (!ok) break;
+                        gm = g2;
+                        stage = 0;
+                    }
+                    cls = un.cold * 2 + un.layer;
+                }
+                const CUtensorMap* mi = M.in[un.layer];
+                if (un.layer == 1) {
+                    // the hidden rows of this token tile must be complete (its weights already stream)
+                    const int32_t* flag = P.ready + un.ready_idx;
+                    const int ready_target = ut.upt[un.cold * 2];   // first-layer units per token tile
+                    if (ld_acquire(flag) < ready_target) {
+                        const uint64_t t0 = global_timer_ns();
+                        while (ld_acquire(flag) < ready_target) {
+                            if (*abort_flag != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
+                                report_timeout(P.status, abort_flag, kSiteHiddenReady);
+                                ok = false;
+                                break;
+                            }
+                        }
+                        if (!ok) break;
+                    }
+                    fence_proxy_async_all();
+                }
+                for (int kb = un.kb0; kb < un.kb1; ++kb) {
+                    if (!mbar_wait(empty_b(stage), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
+                        report_timeout(P.status, abort_flag, kSiteProducerEmpty);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t full = full_b(stage);
+                    const uint32_t b_dst = tiles_u32 + gm.b_base + stage * gm.b_bytes;
+                    mbar_arrive_expect_tx(full, un.nt * 128);
+                    int j = 0;
+                    for (; un.nt - j >= 256; j += 256)
+                        tma_load_2d(b_dst + j * 128, mi + 2, full, kb * kBlockK, un.row0 + j, pol_x);
+                    for (; un.nt - j >= 64; j += 64)
+                        tma_load_2d(b_dst + j * 128, mi + 1, full, kb * kBlockK, un.row0 + j, pol_x);
+                    for (; un.nt - j >= 16; j += 16)
+                        tma_load_2d(b_dst + j * 128, mi, full, kb * kBlockK, un.row0 + j, pol_x);
+                    fill_bits ^= 1u << stage;
+                    if (++stage == gm.nb) stage = 0;
+                }
+            }
+        }
     } else if (warp == 1) {
         // ---- MMA issuer --------------------------------------------------------------
         if (lane == 0) {
-            int stage = 0, cls = -1, stages = 1, stage_bytes = 0, b_off = 0;
-            uint32_t use_bits = 0;      // bit s: parity of the number of uses of stage s
+            int sa = 0, sb = 0, cls = -1;
+            Geom gm = {};
+            uint32_t use_a = 0, use_b = 0;   // bit s: parity of the number of uses of stage s of each ring
             bool ok = true;
             AccCursor acc;
             for (int it = 0; ok; ++it) {
                 const Unit un = pop_unit(it, false);
                 if (un.id < 0) break;
-                if (un.cold * 2 + un.layer != cls &&
-                    (cls < 0 || geom_stage_bytes(un.cold * 2 + un.layer) != stage_bytes ||
-                     geom_b_off(un.cold * 2 + un.layer) != b_off)) {
+                if (un.cold * 2 + un.layer != cls) {
+                    const Geom g2 = geom_of(un.cold * 2 + un.layer);
+                    if (cls < 0 || !same_geom(g2, gm)) {
+                        gm = g2;
+                        sa = 0;
+                        sb = 0;
+                    }
                     cls = un.cold * 2 + un.layer;
-                    stages = geom_stages(cls);
-                    stage_bytes = geom_stage_bytes(cls);
-                    b_off = geom_b_off(cls);
-                    stage = 0;
                 }
                 acc.next(un);
                 const int b = acc.b;
@@ -514,15 +588,16 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                 tc_fence_after_sync();
                 const uint32_t idesc = idesc_bf16_m128(un.nt);
                 for (int kb = un.kb0; kb < un.kb1; ++kb) {
-                    if (!mbar_wait(full_bar(stage), (use_bits >> stage) & 1u, abort_flag, kWaitLimitNs)) {
+                    if (!mbar_wait(full_a(sa), (use_a >> sa) & 1u, abort_flag, kWaitLimitNs) ||
+                        !mbar_wait(full_b(sb), (use_b >> sb) & 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteMmaFull);
                         ok = false;
                         break;
                     }
                     tc_fence_after_sync();
                     if (kb == un.kb0) trace_time(P, it, 3);
-                    const uint32_t a_addr = tiles_u32 + stage * stage_bytes;
-                    const uint64_t b_desc = smem_desc_sw128(a_addr + b_off);
+                    const uint32_t a_addr = tiles_u32 + sa * gm.a_bytes;
+                    const uint64_t b_desc = smem_desc_sw128(tiles_u32 + gm.b_base + sb * gm.b_bytes);
                     for (int t = 0; t < un.tiles; ++t) {      // feature tiles share the token tile
                         const uint64_t a_desc = smem_desc_sw128(a_addr + t * kABytes);
 #pragma unroll
@@ -530,9 +605,12 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(
                             umma_bf16(tmem_base + acc_col(un, b, t), a_desc + 2 * k4, b_desc + 2 * k4, idesc,
                                       (kb != un.kb0) | (k4 != 0));
                     }
-                    umma_commit(empty_bar(stage));   // stage reusable once these MMAs finish
-                    use_bits ^= 1u << stage;
-                    if (++stage == stages) stage = 0;
+                    umma_commit(empty_a(sa));   // both stages reusable once these MMAs finish
+                    umma_commit(empty_b(sb));
+                    use_a ^= 1u << sa;
+                    use_b ^= 1u << sb;
+                    if (++sa == gm.na) sa = 0;
+                    if (++sb == gm.nb) sb = 0;
                 }
                 if (ok) umma_commit(acc_full(b));   // accumulator complete
                 trace_time(P, it, 4);
@@ -810,18 +888,21 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.ready = reinterpret_cast<int32_t*>(base + WsLayout::kTiles);
     P.trace = g_trace;
     P.trace_slots = g_trace_slots;
-    CUtensorMap map_w1, map_w2, map_x, map_h;
-    if (!make_map(&map_w1, W1, static_cast<uint64_t>(p.E) * p.d_ff, p.d_model, kTileRows)) return MONDE_ERR_CUDA;
-    if (!make_map(&map_w2, W2, static_cast<uint64_t>(p.E) * p.d_model, p.d_ff, kTileRows)) return MONDE_ERR_CUDA;
-    if (!make_map(&map_x, x_perm, A, p.d_model, 16)) return MONDE_ERR_CUDA;
-    if (!make_map(&map_h, P.h, A, p.d_ff, 16)) return MONDE_ERR_CUDA;
+    FfnMaps M;
+    const uint32_t in_box[3] = {16, 64, 256};
+    for (int i = 0; i < 2; ++i) {
+        if (!make_map(&M.w[0][i], W1, static_cast<uint64_t>(p.E) * p.d_ff, p.d_model, kTileRows << i)) return MONDE_ERR_CUDA;
+        if (!make_map(&M.w[1][i], W2, static_cast<uint64_t>(p.E) * p.d_model, p.d_ff, kTileRows << i)) return MONDE_ERR_CUDA;
+    }
+    for (int i = 0; i < 3; ++i) {
+        if (!make_map(&M.in[0][i], x_perm, A, p.d_model, in_box[i])) return MONDE_ERR_CUDA;
+        if (!make_map(&M.in[1][i], P.h, A, p.d_ff, in_box[i])) return MONDE_ERR_CUDA;
+    }
     cudaError_t err;
     if (p.act == MONDE_ACT_RELU)
-        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_RELU>, dim3(sm_count()), dim3(kThreads), kSmemBytes, s, map_w1,
-                         map_w2, map_x, map_h, P);
+        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_RELU>, dim3(sm_count()), dim3(kThreads), kSmemBytes, s, M, P);
     else
-        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_GELU_ERF>, dim3(sm_count()), dim3(kThreads), kSmemBytes, s,
-                         map_w1, map_w2, map_x, map_h, P);
+        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_GELU_ERF>, dim3(sm_count()), dim3(kThreads), kSmemBytes, s, M, P);
     if (err != cudaSuccess) return MONDE_ERR_CUDA;
     return launched();
 }
