@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full(b), 1);      // one commit
-            mbar_init(acc_empty(b), 4);     // 4 epilogue warps
+            mbar_init(acc_empty(b), 5);     // 4 epilogue warps + the publisher (keeps it at most one use behind)
             mbar_init(rows_stored(b), 4);   // 4 epilogue warps
         }
         for (int s = 0; s < kQueue; ++s) {
@@ -759,6 +759,10 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 acc.next(un);
                 if (!mbar_wait(rows_stored(acc.b), acc.parity, abort_flag, kWaitLimitNs))
                     break;   // the role that stalled has already reported
+                // Only now may this accumulator buffer be reused: the epilogue cannot signal "rows
+                // stored" for the buffer's next use before this thread has seen the current one
+                // (a waiter that falls two phases behind an mbarrier would wait on the wrong phase).
+                mbar_arrive(acc_empty(acc.b));
                 if (un.layer == 0) {
                     __threadfence();
                     fence_proxy_async_all();
