@@ -81,6 +81,7 @@ struct FfnParams {
     int cold_tile;                // token tile of the cold class
     int pair_mask;                // bit (class * 2 + layer): units of that segment take two feature tiles
     int n_split;                  // K-splits of a cold second-layer unit (1 = none)
+    int split_major;              // ordering of the K-split sub-units (see UnitTable::decode)
     const __nv_bfloat16* b1;
     const __nv_bfloat16* b2;
     __nv_bfloat16* h;
@@ -144,7 +145,7 @@ struct UnitTable {
     int upt[4];                      // units per token tile, by segment (class * 2 + layer)
     int tpu[4];                      // feature tiles per unit, by segment
     int kblocks1, kblocks2;          // 64-wide K blocks of layer 1 (d_model) and layer 2 (d_ff)
-    int n_split, kb_per_split;
+    int n_split, kb_per_split, split_major;
     int seg1, seg2, seg3, total_units;   // list = [hot L1 | hot L2 | cold L1 | cold L2 (split)]
 
     __device__ __forceinline__ Unit decode(int u) const {
@@ -157,21 +158,64 @@ struct UnitTable {
         else { r.cold = 1; r.layer = 1; v = u - seg3; }
         r.split = 0;
         r.n_split = 1;
-        if (r.cold && r.layer) {
-            r.n_split = n_split;
-            r.split = v % n_split;
-            v /= n_split;
-        }
         const int sgm = r.cold * 2 + r.layer;
-        const int ntl = upt[sgm];
         const int lo_entry = r.cold ? n_hot : 0;
         const int tt_base = tt_prefix[lo_entry];
-        int lo = lo_entry, hi = (r.cold ? n_all : n_hot) - 1;      // largest entry with block start <= v
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if ((tt_prefix[mid] - tt_base) * ntl <= v) lo = mid; else hi = mid - 1;
+        int lo, local;
+        if (r.cold && r.layer && n_split > 1 && split_major) {
+            // K-split segment, split index slowest over the whole segment: every expert's sub-units 0,
+            // then 1, ..., and the finishing sub-units (S-1) at the very end of the list, where they
+            // find their partial tiles long done and make a short tail.
+            r.n_split = n_split;
+            const int per_split = (total_units - seg3) / n_split;
+            r.split = v / per_split;
+            v -= r.split * per_split;
+            const int ntl = upt[3];
+            lo = lo_entry;
+            int hi = n_all - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if ((tt_prefix[mid] - tt_base) * ntl <= v) lo = mid; else hi = mid - 1;
+            }
+            local = v - (tt_prefix[lo] - tt_base) * ntl;
+        } else if (r.cold && r.layer && n_split > 1) {
+            // K-split segment, in slots: slot j holds the partial sub-units (splits 0..S-2, split
+            // index slowest) of cold expert j followed by the finishing sub-units (split S-1) of
+            // expert j-1.  A finisher is thus taken a good fraction of a scheduling round after the
+            // partial tiles it adds (it does not wait for them) yet soon enough to find them in L2.
+            r.n_split = n_split;
+            const int n = n_all - n_hot;
+            const int pm = upt[3] * (n_split - 1), fm = upt[3];
+            auto before = [&](int j) {
+                return pm * (tt_prefix[lo_entry + min(j, n)] - tt_base) + fm * (tt_prefix[lo_entry + max(j - 1, 0)] - tt_base);
+            };
+            int a = 0, b = n;                              // largest slot with before(slot) <= v
+            while (a < b) {
+                const int mid = (a + b + 1) >> 1;
+                if (before(mid) <= v) a = mid; else b = mid - 1;
+            }
+            local = v - before(a);
+            const int partial_units = a < n ? pm * tt[lo_entry + a] : 0;
+            if (local < partial_units) {
+                lo = lo_entry + a;
+                const int per_split = tt[lo] * upt[3];
+                r.split = local / per_split;
+                local -= r.split * per_split;
+            } else {
+                lo = lo_entry + a - 1;
+                local -= partial_units;
+                r.split = n_split - 1;
+            }
+        } else {
+            const int ntl = upt[sgm];
+            lo = lo_entry;
+            int hi = (r.cold ? n_all : n_hot) - 1;      // largest entry with block start <= v
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if ((tt_prefix[mid] - tt_base) * ntl <= v) lo = mid; else hi = mid - 1;
+            }
+            local = v - (tt_prefix[lo] - tt_base) * ntl;
         }
-        const int local = v - (tt_prefix[lo] - tt_base) * ntl;
         const int tok = local % tt[lo];
         const int ntile = local / tt[lo];
         r.e = e[lo];
@@ -355,6 +399,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     ut.kblocks1 = P.d_model / kBlockK;
     ut.kblocks2 = P.d_ff / kBlockK;
     ut.n_split = P.n_split;
+    ut.split_major = P.split_major;
     ut.kb_per_split = (ut.kblocks2 + P.n_split - 1) / P.n_split;
     ut.seg1 = tt_hot * ut.upt[0];
     ut.seg2 = ut.seg1 + tt_hot * ut.upt[1];
@@ -887,6 +932,11 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.pair_mask = 0xC | (p.d_model >= 1536 ? 0x3 : 0);
     const WsLayout L = ws_layout(p);
     P.n_split = L.n_split;
+    // Finishing sub-units at the very end of the list give the shortest tail (Switch-Base-sized
+    // layer: 152 -> 144 us) but their partial tiles must survive in L2 while the rest of the
+    // cold second-layer weights stream through; with gigabytes of weights they do not (NLLB-sized
+    // layer: 1.38 -> 1.41 ms), and the expert-by-expert order is used instead.
+    P.split_major = 4.0 * p.E * p.d_model * static_cast<double>(p.d_ff) <= 1.0e9;
     P.part_done = reinterpret_cast<int32_t*>(base + L.part_done_off);
     P.partials = reinterpret_cast<float*>(base + L.partials_off);
     P.ready = reinterpret_cast<int32_t*>(base + WsLayout::kTiles);
