@@ -207,6 +207,9 @@ def run_ours(args, w):
             ev[0].record(stream)
         B.monde_route(p, d["x"], d["Wg"], d["bg"], buf.topk_idx, buf.topk_w, buf.counts, buf.offsets, buf.cls,
                       buf.hot_ids, buf.cold_ids, buf.n_hot_cold, None, buf.ws)
+        if args.policy == "top_h":     # the paper's placement rule replaces the threshold classes
+            B.monde_classify_top_h(p, buf.counts, args.alpha, args.bw_hot, args.bw_cold, buf.cls, buf.hot_ids,
+                                   buf.cold_ids, buf.n_hot_cold)
         if ev is not None:
             ev[1].record(stream)
         B.monde_permute(p, d["x"], buf.topk_idx, buf.offsets, buf.perm, buf.inv_perm, buf.x_perm, buf.ws)
@@ -225,6 +228,7 @@ def run_ours(args, w):
         layer()
     B.monde_poll_device_status(buf.ws)
     counts = buf.counts.cpu().numpy()
+    n_hot_used = int(buf.n_hot_cold.cpu()[0])
 
     # ---- timed region: device-resident inputs --------------------------------------
     # Events bracket whole steps only: the four calls overlap through programmatic dependent
@@ -330,7 +334,9 @@ def run_ours(args, w):
                      "ffn": ffn_ms, "combine": statistics.mean(call_ms[3])},
         "calls_ms_sum": sum(statistics.mean(c) for c in call_ms),
         "layer_hbm_floor_ms": layer_floor_ms, "layer_roofline_frac": layer_floor_ms / ms_per_step,
-        "routing": {"active": int((counts > 0).sum()), "hot": int((counts >= p.hot_threshold).sum()),
+        "policy": args.policy if args.policy == "threshold" else
+        f"top_h alpha={args.alpha} bw_hot={args.bw_hot} bw_cold={args.bw_cold}",
+        "routing": {"active": int((counts > 0).sum()), "hot": n_hot_used,
                     "max_count": int(counts.max()), "assignments": int(counts.sum())},
         "wall_s_timed_region": wall,
     }
@@ -347,6 +353,11 @@ def main():
     ap.add_argument("--workload", default="C1", choices=["C1", "C2", "C3"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--policy", default="threshold", choices=["threshold", "top_h"],
+                    help="hot/cold rule: count >= hot_threshold, or the paper's top-H rule (Eq. 6)")
+    ap.add_argument("--alpha", type=float, default=1.0, help="Eq. 6 tuning factor (top_h)")
+    ap.add_argument("--bw-hot", type=float, default=3.9, help="TB/s at which the hot tiling consumes weights (top_h)")
+    ap.add_argument("--bw-cold", type=float, default=7.0, help="TB/s at which the cold tiling streams weights (top_h)")
     args = ap.parse_args()
     w = S.config(args.workload)
     if args.impl == "reference":

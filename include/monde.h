@@ -97,6 +97,25 @@ int monde_route(const monde_problem* p, const void* x, const void* Wg, const flo
                 uint8_t* cls, int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold,
                 float* probs, void* ws, size_t ws_bytes, void* stream);
 
+/* Hot / cold lists by the paper's own placement rule instead of a count threshold; run it after
+ * monde_route to overwrite cls / hot_ids / cold_ids / n_hot_cold (counts, offsets and the
+ * permutation do not depend on the classes).
+ * Paper: Section 3.3, Eq. 3-6.  The H experts with the most tokens go to the engine whose cost is
+ * fetching their weights (bandwidth BW_a; the GPU behind PCIe in the paper, the hot class here),
+ * the rest to the engine that streams them in place (bandwidth BW_b; the near-data device in the
+ * paper, the cold class here), with
+ *     H = alpha * BW_a / (BW_b + BW_a) * Expert_Activ                                  (Eq. 6)
+ * Expert_Activ = experts with at least one token (Eq. 5).  H is rounded down and clamped to
+ * [0, Expert_Activ]; "most compute-intensive" = most tokens; equal counts: the smaller id is hotter;
+ * experts without tokens stay class 0.  alpha is the paper's tuning factor (its auto-tuner tries
+ * H, H+1, H+2 on recent batches and keeps the fastest).
+ * in : counts [E] (device); alpha >= 0, bw_hot_feed (BW_a) > 0, bw_cold_feed (BW_b) > 0 (any common unit)
+ * out: cls [E], hot_ids [E], cold_ids [E], n_hot_cold [2] as in monde_route
+ */
+int monde_classify_top_h(const monde_problem* p, const int32_t* counts, double alpha, double bw_hot_feed,
+                         double bw_cold_feed, uint8_t* cls, int32_t* hot_ids, int32_t* cold_ids,
+                         int32_t* n_hot_cold, void* stream);
+
 /* Stable permutation of assignments into expert-contiguous order and row gather.
  * Paper: Section 2.1 (tokens routed to experts, later re-organised into the original
  * order); Section 4.1 (drop-less, padding-less routing: no capacity, no padded slot).

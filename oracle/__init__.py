@@ -121,6 +121,19 @@ def combine(y_perm, inv_perm, topk_w):
     return out
 
 
+def classify_top_h(counts, alpha: float, bw_a: float, bw_b: float):
+    """Hot / cold lists by the paper's top-H rule (Section 3.3, Eq. 6) instead of a threshold."""
+    counts = np.ascontiguousarray(counts, np.int32)
+    E = counts.shape[0]
+    r = SimpleNamespace(cls=np.zeros(E, np.uint8), hot_ids=np.full(E, -1, np.int32),
+                        cold_ids=np.full(E, -1, np.int32), n_hot_cold=np.zeros(2, np.int32),
+                        H=np.zeros(1, np.int32))
+    lib().oracle_classify_top_h(E, _p(counts), ctypes.c_double(alpha), ctypes.c_double(bw_a), ctypes.c_double(bw_b),
+                                _p(r.cls), _p(r.hot_ids), _p(r.cold_ids), _p(r.n_hot_cold), _p(r.H))
+    r.H = int(r.H[0])
+    return r
+
+
 def experts_of_rows(offsets: np.ndarray) -> np.ndarray:
     """Expert id of every row of the expert-contiguous buffer."""
     return np.repeat(np.arange(offsets.shape[0] - 1, dtype=np.int32), np.diff(offsets)).astype(np.int32)

@@ -211,3 +211,39 @@ void oracle_combine(int T, int d, int k, const double* y_perm, const int32_t* in
 }
 
 }  // extern "C"
+
+extern "C" {
+
+// The paper's own placement rule (Section 3.3, Eq. 3-6): with Expert_Activ the number of experts
+// that received at least one token (Eq. 5), the H experts with the most tokens go to the engine
+// that must first fetch their weights (here: the hot class) and the rest to the engine that
+// streams them in place (the cold class), where
+//     H = alpha * BW_a / (BW_b + BW_a) * Expert_Activ            (Eq. 6)
+// BW_a is the bandwidth that feeds the hot side (PCIe in the paper), BW_b the one that feeds the
+// cold side (the memory device's), alpha the tuning factor.  Readings: H is rounded down and
+// clamped to [0, Expert_Activ]; "most compute-intensive" = most tokens, equal counts -> the
+// smaller expert id is hotter; experts without tokens stay inactive (class 0).
+void oracle_classify_top_h(int E, const int32_t* counts, double alpha, double bw_a, double bw_b,
+                           uint8_t* cls, int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold,
+                           int32_t* h_out) {
+    int active = 0;
+    for (int e = 0; e < E; ++e) active += counts[e] > 0;
+    double h_real = alpha * bw_a / (bw_b + bw_a) * static_cast<double>(active);
+    int H = h_real <= 0.0 ? 0 : static_cast<int>(std::floor(h_real));
+    if (H > active) H = active;
+    std::vector<int> order;
+    for (int e = 0; e < E; ++e) if (counts[e] > 0) order.push_back(e);
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return counts[a] > counts[b]; });
+    for (int e = 0; e < E; ++e) cls[e] = counts[e] > 0 ? 1 : 0;
+    for (int r = 0; r < H; ++r) cls[order[r]] = 2;
+    int nh = 0, nc = 0;
+    for (int e = 0; e < E; ++e) {
+        if (cls[e] == 2) hot_ids[nh++] = e;
+        else if (cls[e] == 1) cold_ids[nc++] = e;
+    }
+    n_hot_cold[0] = nh;
+    n_hot_cold[1] = nc;
+    if (h_out) *h_out = H;
+}
+
+}  // extern "C"

@@ -16,7 +16,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmonde.so")
 
-SYMBOLS = ("monde_workspace_bytes", "monde_status_string", "monde_route", "monde_permute",
+SYMBOLS = ("monde_workspace_bytes", "monde_status_string", "monde_route", "monde_classify_top_h", "monde_permute",
            "monde_moe_ffn_fwd", "monde_moe_ffn_fwd_static_ws", "monde_combine", "monde_poll_device_status",
            "monde_kernel_launches")
 
@@ -56,6 +56,9 @@ def lib() -> ctypes.CDLL:
         L.monde_route.restype = ctypes.c_int
         L.monde_route.argtypes = [pp, vp, vp, f32p, i32p, f32p, i32p, i32p, vp, i32p, i32p, i32p, f32p,
                                   vp, ctypes.c_size_t, vp]
+        L.monde_classify_top_h.restype = ctypes.c_int
+        L.monde_classify_top_h.argtypes = [pp, i32p, ctypes.c_double, ctypes.c_double, ctypes.c_double, vp, i32p, i32p,
+                                           i32p, vp]
         L.monde_permute.restype = ctypes.c_int
         L.monde_permute.argtypes = [pp, vp, i32p, i32p, i32p, i32p, vp, vp, ctypes.c_size_t, vp]
         L.monde_moe_ffn_fwd.restype = ctypes.c_int
@@ -110,6 +113,14 @@ def monde_route(p, x, Wg, bg, topk_idx, topk_w, counts, offsets, cls, hot_ids, c
         ctypes.byref(cp), _ptr(x), _ptr(Wg), _ptr(bg), _ptr(topk_idx), _ptr(topk_w), _ptr(counts),
         _ptr(offsets), _ptr(cls), _ptr(hot_ids), _ptr(cold_ids), _ptr(n_hot_cold), _ptr(probs),
         _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def monde_classify_top_h(p, counts, alpha, bw_hot_feed, bw_cold_feed, cls, hot_ids, cold_ids, n_hot_cold,
+                         stream=None) -> None:
+    cp = c_problem(p)
+    _check("monde_classify_top_h", lib().monde_classify_top_h(
+        ctypes.byref(cp), _ptr(counts), float(alpha), float(bw_hot_feed), float(bw_cold_feed), _ptr(cls),
+        _ptr(hot_ids), _ptr(cold_ids), _ptr(n_hot_cold), _stream(stream)))
 
 
 def monde_permute(p, x, topk_idx, offsets, perm, inv_perm, x_perm, ws, stream=None) -> None:

@@ -91,6 +91,19 @@ int monde_route(const monde_problem* p, const void* x, const void* Wg, const flo
                         ticket, s);
 }
 
+int monde_classify_top_h(const monde_problem* p, const int32_t* counts, double alpha, double bw_hot_feed,
+                         double bw_cold_feed, uint8_t* cls, int32_t* hot_ids, int32_t* cold_ids,
+                         int32_t* n_hot_cold, void* stream) {
+    int st = check_problem(p);
+    if (st != MONDE_OK) return st;
+    if (!counts || !cls || !hot_ids || !cold_ids || !n_hot_cold) return MONDE_ERR_INVALID_ARG;
+    if (!(alpha >= 0.0) || !(bw_hot_feed > 0.0) || !(bw_cold_feed > 0.0)) return MONDE_ERR_INVALID_ARG;
+    if ((st = check_arch()) != MONDE_OK) return st;
+    const double share = alpha * bw_hot_feed / (bw_cold_feed + bw_hot_feed);
+    return launch_classify_top_h(*p, share, counts, cls, hot_ids, cold_ids, n_hot_cold,
+                                 static_cast<cudaStream_t>(stream));
+}
+
 int monde_permute(const monde_problem* p, const void* x, const int32_t* topk_idx,
                   const int32_t* offsets, int32_t* perm, int32_t* inv_perm, void* x_perm,
                   void* ws, size_t ws_bytes, void* stream) {

@@ -126,6 +126,8 @@ __device__ __forceinline__ float apply_act(float v, int act) {
 int launch_route(const monde_problem& p, const void* x, const void* Wg, const float* bg,
                  int32_t* topk_idx, float* topk_w, float* probs, int32_t* counts, int32_t* offsets, uint8_t* cls,
                  int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, int32_t* ticket, cudaStream_t s);
+int launch_classify_top_h(const monde_problem& p, double share, const int32_t* counts, uint8_t* cls,
+                          int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, cudaStream_t s);
 int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_idx, const int32_t* offsets,
                    int32_t* perm, int32_t* inv_perm, void* x_perm, cudaStream_t s);
 int launch_combine(const monde_problem& p, const void* y_perm, const int32_t* inv_perm,

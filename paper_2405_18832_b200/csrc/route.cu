@@ -311,6 +311,62 @@ int launch_route_mma(const monde_problem& p, const void* x, const void* Wg, cons
     return MONDE_OK;
 }
 
+// The paper's own placement rule (Section 3.3, Eq. 3-6): the H experts with the most tokens are
+// hot, H = floor(share * Expert_Activ) with share = alpha * BW_a / (BW_b + BW_a) and Expert_Activ
+// the number of experts with at least one token (Eq. 5); equal counts: the smaller id is hotter.
+// One CTA of 256 threads: thread e ranks expert e against all others.
+__global__ void __launch_bounds__(kMaxExperts) classify_top_h_kernel(
+        int E, double share, const int32_t* __restrict__ counts, uint8_t* __restrict__ cls,
+        int32_t* __restrict__ hot_ids, int32_t* __restrict__ cold_ids, int32_t* __restrict__ n_hot_cold) {
+    __shared__ int s_cnt[kMaxExperts];
+    __shared__ int s_cls[kMaxExperts];
+    __shared__ int s_active;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int e = threadIdx.x;
+    if (e == 0) s_active = 0;
+    s_cnt[e] = e < E ? counts[e] : 0;
+    __syncthreads();
+    const int c = s_cnt[e];
+    if (c > 0) atomicAdd(&s_active, 1);
+    int rank = 0;
+    for (int o = 0; o < E; ++o) rank += (s_cnt[o] > c) || (s_cnt[o] == c && o < e);
+    __syncthreads();
+    const double h_real = share * static_cast<double>(s_active);
+    int H = h_real <= 0.0 ? 0 : static_cast<int>(floor(h_real));
+    H = min(H, s_active);
+    const int k = c > 0 ? (rank < H ? 2 : 1) : 0;
+    s_cls[e] = k;
+    if (e < E) cls[e] = static_cast<uint8_t>(k);
+    __syncthreads();
+    if (threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;       // lane owns experts [lane*8, lane*8+8): ascending compaction
+    int nh = 0, nc = 0;
+#pragma unroll
+    for (int i = 0; i < kSlots; ++i) {
+        nh += s_cls[lane * kSlots + i] == 2;
+        nc += s_cls[lane * kSlots + i] == 1;
+    }
+    int ph = nh, pc = nc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, ph, o);
+        const int b = __shfl_up_sync(0xffffffffu, pc, o);
+        if (lane >= o) { ph += a; pc += b; }
+    }
+    int ih = ph - nh, ic = pc - nc;
+#pragma unroll
+    for (int i = 0; i < kSlots; ++i) {
+        const int x = lane * kSlots + i;
+        if (s_cls[x] == 2) hot_ids[ih++] = x;
+        else if (s_cls[x] == 1) cold_ids[ic++] = x;
+    }
+    if (lane == 31) {
+        n_hot_cold[0] = ph;
+        n_hot_cold[1] = pc;
+    }
+}
+
 }  // namespace
 
 int launch_route(const monde_problem& p, const void* x, const void* Wg, const float* bg,
@@ -334,6 +390,13 @@ int launch_route(const monde_problem& p, const void* x, const void* Wg, const fl
             p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const float*>(x),
             static_cast<const float*>(Wg), bg, topk_idx, topk_w, probs, hist);
     }
+    return launched();
+}
+
+int launch_classify_top_h(const monde_problem& p, double share, const int32_t* counts, uint8_t* cls,
+                          int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, cudaStream_t s) {
+    launch_pdl(classify_top_h_kernel, dim3(1), dim3(kMaxExperts), 0, s, p.E, share, counts, cls, hot_ids, cold_ids,
+               n_hot_cold);
     return launched();
 }
 

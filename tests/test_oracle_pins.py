@@ -278,3 +278,38 @@ def test_combine_is_a_weighted_gather():
     out = oracle.combine(y, inv, w)
     want = np.einsum("tk,tkd->td", w, y[inv].reshape(T, k, d))
     np.testing.assert_allclose(out, want, rtol=1e-14)
+
+
+# ---------------------------------------------------------------- top-H placement (Section 3.3, Eq. 6)
+
+def test_top_h_matches_eq6_worked_by_hand():
+    # 10 active of 12 experts; BW_a = 32, BW_b = 96 -> share 32/128 = 1/4.
+    counts = np.array([5, 0, 9, 1, 1, 7, 2, 0, 3, 4, 6, 8], np.int32)
+    r = oracle.classify_top_h(counts, 1.0, 32.0, 96.0)
+    assert r.H == 2                                   # floor(1 * 0.25 * 10) = 2
+    assert r.hot_ids[:2].tolist() == [2, 11]          # counts 9 and 8
+    assert r.n_hot_cold.tolist() == [2, 8] and r.cls[1] == 0 and r.cls[7] == 0
+    assert oracle.classify_top_h(counts, 2.0, 32.0, 96.0).H == 5      # alpha scales H
+    assert oracle.classify_top_h(counts, 1.3, 32.0, 96.0).H == 3      # floor(3.25)
+    assert oracle.classify_top_h(counts, 0.0, 32.0, 96.0).n_hot_cold.tolist() == [0, 10]
+    assert oracle.classify_top_h(counts, 100.0, 32.0, 96.0).n_hot_cold.tolist() == [10, 0]   # clamped to Expert_Activ
+
+
+def test_top_h_ties_go_to_the_smaller_expert_id_and_balances_the_two_workflows():
+    counts = np.array([4, 4, 4, 4, 0, 4, 4], np.int32)
+    r = oracle.classify_top_h(counts, 1.0, 1.0, 1.0)          # H = floor(0.5 * 6) = 3
+    assert r.hot_ids[:3].tolist() == [0, 1, 2] and r.cold_ids[:3].tolist() == [3, 5, 6]
+    # Eq. 4 with equal expert sizes: t_PM ~ H / BW_a, t_MD ~ (Activ - H) / BW_b are balanced by Eq. 6
+    active, bw_a, bw_b = 40, 3.0, 5.0
+    c = np.arange(1, active + 1, dtype=np.int32)
+    H = oracle.classify_top_h(c, 1.0, bw_a, bw_b).H
+    assert abs(H / bw_a - (active - H) / bw_b) <= 1.0 / bw_a + 1.0 / bw_b
+
+
+def test_top_h_equals_the_threshold_rule_at_the_matching_threshold():
+    rng = np.random.default_rng(12)
+    counts = rng.permutation(np.arange(0, 40)).astype(np.int32)      # distinct counts, one zero
+    r = oracle.classify_top_h(counts, 1.0, 1.0, 3.0)                 # H = floor(39 / 4) = 9
+    theta = np.sort(counts)[::-1][r.H - 1]
+    cls = np.where(counts == 0, 0, np.where(counts >= theta, 2, 1))
+    np.testing.assert_array_equal(r.cls, cls)
