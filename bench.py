@@ -307,7 +307,8 @@ def run_ours(args, w):
                 "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
                 "algorithmic_bytes": bytes_ffn, "ms": ffn_ms,
                 "timing": "CUDA events around the call on its stream, per-call pass of the same K steps",
-                "tflops": ffn_flops(p, counts) / (ffn_ms * 1e-3) / 1e12}
+                "tflops": ffn_flops(p, counts) / (ffn_ms * 1e-3) / 1e12,
+                "tensor_frac_of_measured_burst": ffn_flops(p, counts) / (ffn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
     layer_floor_ms = (bytes_ffn + (2 * p.A + 2 * p.T) * p.d_model * p.elem_bytes + p.T * p.d_model * p.elem_bytes) \
         / (peaks["hbm_gbs"] * 1e9) * 1e3
 
@@ -350,7 +351,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="C1", choices=["C1", "C2", "C3"])
+    ap.add_argument("--workload", default="C1",
+                    help="C1 (default), C2, C3, or a crossover-sweep point C4:<d_model>:<T>:<zipf alpha>:<threshold>")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--policy", default="threshold", choices=["threshold", "top_h"],
@@ -359,7 +361,11 @@ def main():
     ap.add_argument("--bw-hot", type=float, default=3.9, help="TB/s at which the hot tiling consumes weights (top_h)")
     ap.add_argument("--bw-cold", type=float, default=7.0, help="TB/s at which the cold tiling streams weights (top_h)")
     args = ap.parse_args()
-    w = S.config(args.workload)
+    if args.workload.startswith("C4:"):
+        _, d_model, T, zipf, theta = args.workload.split(":")
+        w = S.sweep_point(int(d_model), int(T), float(zipf), int(theta))
+    else:
+        w = S.config(args.workload)
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -155,6 +155,8 @@ def config(name: str) -> Workload:
         return Workload("C2", Problem(32, 1024, 4096, 128, 1, 16, 0, "bf16", "relu"), 0.0, 2)
     if name == "C3":   # NLLB-MoE-like layer
         return Workload("C3", Problem(2048, 2048, 8192, 128, 2, 32, 1, "bf16", "relu"), 1.0, 3)
+    if name == "HOTPROBE":   # compute-bound probe of the hot tiling: 8 experts x ~2048 tokens, NLLB-sized FFN
+        return Workload("HOTPROBE", Problem(16384, 2048, 8192, 8, 1, 32, 0, "bf16", "relu"), 0.0, 5)
     raise KeyError(name)
 
 

@@ -131,3 +131,13 @@ def test_crossover_sweep_sampled_parity(d_model, n_sample):
                     P.check_routing(wt.problem, g, buf)
                     # same experts, same rows: only the class, hence the tiling, may differ
                     P.check_close(f"out theta={theta}", P.widen(buf.out), P.widen(first.out), "bf16")
+
+
+def test_compute_bound_probe_sampled_parity():
+    # 8 experts x ~2048 tokens each: every expert hot, many 256-token tiles per expert
+    w = S.config("HOTPROBE")
+    g = S.generate(w, with_weights=False)
+    dev = P.to_device(g)
+    dev.update({k: v for k, v in S.generate(w, weights_device="cuda").items() if k in ("W1", "W2", "b1", "b2")})
+    r = P.check_sampled(w, g, dev, n_tokens=48)
+    assert r.route.n_hot_cold.tolist() == [8, 0]
