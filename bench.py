@@ -171,6 +171,43 @@ def run_reference(args, w):
         "gpu_launches": 0}))
 
 
+def dist_setup(backend: str, device=None):
+    """Joins the process group that torchrun describes in the environment (one rank per GPU).
+    Returns (dist module or None, rank, world, local_rank)."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world == 1:
+        return None, rank, world, local
+    import torch.distributed as dist
+    if backend == "nccl":
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        dist.init_process_group(backend)
+    return dist, rank, world, local
+
+
+def max_over_ranks(dist, value: float, device="cpu") -> float:
+    """Slowest rank's device time: what a job of independent replicas has to wait for."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_workload(w, rank: int, world: int):
+    """Every replica gets its own batch (same layer, different tokens)."""
+    if world == 1:
+        return w
+    import dataclasses
+    return dataclasses.replace(w, seed=w.seed + 1000 * rank)
+
+
+def aggregate_tokens_per_s(tokens_per_step_per_gpu: int, world: int, ms_per_step: float) -> float:
+    return world * tokens_per_step_per_gpu / (ms_per_step * 1e-3)
+
+
 def workload_config(w):
     p = w.problem
     return {"workload": f"{w.name}: E={p.E} top-{p.top_k} d_model={p.d_model} d_ff={p.d_ff} T={p.T} {p.dtype} "
@@ -182,19 +219,11 @@ def workload_config(w):
 
 def run_ours(args, w):
     from paper_2405_18832_b200 import binding as B
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    torch.cuda.set_device(local)
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    dist, rank, world, local = dist_setup("nccl")
     dev = torch.device("cuda", local)
     p = w.problem
-    if world > 1:   # every replica gets its own batch
-        import dataclasses
-        w = dataclasses.replace(w, seed=w.seed + 1000 * rank)
+    w = replica_workload(w, rank, world)
     g = generate_inputs(w, dev)
     d = {k: (None if v is None else v.to(dev)) for k, v in g.items()}
     buf = B.LayerBuffers(p, device=dev)
@@ -255,13 +284,9 @@ def run_ours(args, w):
     clocks = sampler.stop()
     sys.setswitchinterval(switch_interval)
     B.monde_poll_device_status(buf.ws)
-    total_ms = sum(a.elapsed_time(b) for a, b in events)
-    tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-    total_ms = float(tt.item())
+    total_ms = max_over_ranks(dist, sum(a.elapsed_time(b) for a, b in events), dev)
     ms_per_step = total_ms / args.steps
-    value = world * p.T / (ms_per_step * 1e-3)
+    value = aggregate_tokens_per_s(p.T, world, ms_per_step)
 
     # ---- per-call pass: the same K steps again with an event between the calls, which gives
     # each call's own duration (and the dominant kernel's, for the roofline) at the price of
@@ -286,11 +311,8 @@ def run_ours(args, w):
         B.moe_ffn_layer_forward_host(p, x_host, out_host, d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"], buf)
         b.record(stream)
     torch.cuda.synchronize()
-    e2e_ms = sum(a.elapsed_time(b) for a, b in e2e_ev)
-    te = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_value = world * p.T / (float(te.item()) / args.steps * 1e-3)
+    e2e_ms = max_over_ranks(dist, sum(a.elapsed_time(b) for a, b in e2e_ev), dev)
+    e2e_value = aggregate_tokens_per_s(p.T, world, e2e_ms / args.steps)
     assert torch.equal(out_host, buf.out.cpu())
 
     if rank != 0:
