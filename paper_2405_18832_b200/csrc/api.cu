@@ -114,7 +114,8 @@ int monde_permute(const monde_problem* p, const void* x, const int32_t* topk_idx
     if (!aligned16(x) || !aligned16(x_perm)) return MONDE_ERR_INVALID_ARG;
     if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
     if ((st = check_arch()) != MONDE_OK) return st;
-    return launch_permute(*p, x, topk_idx, offsets, perm, inv_perm, x_perm, static_cast<cudaStream_t>(stream));
+    int32_t* scratch = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + WsLayout::kHidden);
+    return launch_permute(*p, x, topk_idx, offsets, perm, inv_perm, x_perm, scratch, static_cast<cudaStream_t>(stream));
 }
 
 int monde_moe_ffn_fwd(const monde_problem* p, const void* x_perm,

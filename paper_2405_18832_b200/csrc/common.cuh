@@ -128,8 +128,10 @@ int launch_route(const monde_problem& p, const void* x, const void* Wg, const fl
                  int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, int32_t* ticket, cudaStream_t s);
 int launch_classify_top_h(const monde_problem& p, double share, const int32_t* counts, uint8_t* cls,
                           int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, cudaStream_t s);
+// `scratch`: at least ceil(A / 2048) * E int32 of workspace that is dead during the call (the hidden-
+// activation region serves: the expert FFN rewrites it before reading it); used when A > 8192.
 int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_idx, const int32_t* offsets,
-                   int32_t* perm, int32_t* inv_perm, void* x_perm, cudaStream_t s);
+                   int32_t* perm, int32_t* inv_perm, void* x_perm, int32_t* scratch, cudaStream_t s);
 int launch_combine(const monde_problem& p, const void* y_perm, const int32_t* inv_perm,
                    const float* topk_w, void* out, cudaStream_t s);
 

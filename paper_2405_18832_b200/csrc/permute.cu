@@ -17,11 +17,45 @@ constexpr int kRowsPerWarp = kChunk / (kThreads / 32);
 // the kernel single-pass and free of inter-CTA ordering.  Small chunks give many CTAs and
 // every warp keeps the loads of its four rows in flight together, which is what matters
 // for a decode-sized batch where the whole gather is a few dozen rows.
+// Large batches: the recount of earlier assignments would grow quadratically, so it is cut at
+// super-chunk boundaries.  `super_before` [n_super][E] holds, per expert, the number of assignments in
+// all earlier super-chunks (two small kernels below build it); a CTA then recounts only from the start
+// of its own super-chunk.  Null for small batches: recount from assignment 0.
+constexpr int kSuper = 2048;         // assignments per super-chunk
+constexpr int kTwoLevelFrom = 8192;  // batches with more assignments take the two-level path
+
+__global__ void __launch_bounds__(256) super_histogram_kernel(int A, int E, const int32_t* __restrict__ topk_idx,
+                                                              int32_t* __restrict__ super_before) {
+    __shared__ int hist[kMaxExperts];
+    pdl_launch_dependents();
+    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) hist[e] = 0;
+    __syncthreads();
+    pdl_wait();
+    const int first = blockIdx.x * kSuper;
+    for (int a = first + threadIdx.x; a < min(A, first + kSuper); a += blockDim.x) atomicAdd(&hist[topk_idx[a]], 1);
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) super_before[static_cast<size_t>(blockIdx.x) * E + e] = hist[e];
+}
+
+// In place: counts per super-chunk -> exclusive prefix over super-chunks, one thread per expert.
+__global__ void __launch_bounds__(256) super_scan_kernel(int n_super, int E, int32_t* __restrict__ super_before) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int e = threadIdx.x;
+    if (e >= E) return;
+    int running = 0;
+    for (int s = 0; s < n_super; ++s) {
+        const int c = super_before[static_cast<size_t>(s) * E + e];
+        super_before[static_cast<size_t>(s) * E + e] = running;
+        running += c;
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
         int A, int E, int k, int d, const T* __restrict__ x, const int32_t* __restrict__ topk_idx,
-        const int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
-        T* __restrict__ x_perm) {
+        const int32_t* __restrict__ offsets, const int32_t* __restrict__ super_before,
+        int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, T* __restrict__ x_perm) {
     __shared__ int before[kMaxExperts];   // assignments to e in earlier chunks
     __shared__ int row_pos[kChunk];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -30,7 +64,11 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
     for (int e = tid; e < kMaxExperts; e += kThreads) before[e] = 0;
     __syncthreads();
     pdl_wait();
-    for (int a = tid; a < first; a += kThreads) atomicAdd(&before[topk_idx[a]], 1);
+    const int recount_from = super_before != nullptr ? (first / kSuper) * kSuper : 0;
+    if (super_before != nullptr)
+        for (int e = tid; e < E; e += kThreads) before[e] = super_before[static_cast<size_t>(first / kSuper) * E + e];
+    __syncthreads();
+    for (int a = recount_from + tid; a < first; a += kThreads) atomicAdd(&before[topk_idx[a]], 1);
     __syncthreads();
     if (warp == 0) {
         const int a = first + lane;
@@ -98,16 +136,24 @@ __global__ void __launch_bounds__(256) combine_kernel(
 }  // namespace
 
 int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_idx, const int32_t* offsets,
-                   int32_t* perm, int32_t* inv_perm, void* x_perm, cudaStream_t s) {
+                   int32_t* perm, int32_t* inv_perm, void* x_perm, int32_t* scratch, cudaStream_t s) {
     const int A = p.T * p.top_k;
     const int grid = (A + kChunk - 1) / kChunk;
+    int32_t* super_before = nullptr;
+    if (A > kTwoLevelFrom) {
+        const int n_super = (A + kSuper - 1) / kSuper;
+        super_before = scratch;      // n_super * E int32
+        launch_pdl(super_histogram_kernel, dim3(n_super), dim3(256), 0, s, A, p.E, topk_idx, super_before);
+        launch_pdl(super_scan_kernel, dim3(1), dim3(256), 0, s, n_super, p.E, super_before);
+        count_launches(2);
+    }
     if (p.dtype == MONDE_BF16)
         launch_pdl(permute_gather_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), 0, s,
-            A, p.E, p.top_k, p.d_model, static_cast<const __nv_bfloat16*>(x), topk_idx, offsets, perm,
+            A, p.E, p.top_k, p.d_model, static_cast<const __nv_bfloat16*>(x), topk_idx, offsets, super_before, perm,
             inv_perm, static_cast<__nv_bfloat16*>(x_perm));
     else
         launch_pdl(permute_gather_kernel<float>, dim3(grid), dim3(kThreads), 0, s,
-            A, p.E, p.top_k, p.d_model, static_cast<const float*>(x), topk_idx, offsets, perm, inv_perm,
+            A, p.E, p.top_k, p.d_model, static_cast<const float*>(x), topk_idx, offsets, super_before, perm, inv_perm,
             static_cast<float*>(x_perm));
     return launched();
 }

@@ -141,3 +141,14 @@ def test_compute_bound_probe_sampled_parity():
     dev.update({k: v for k, v in S.generate(w, weights_device="cuda").items() if k in ("W1", "W2", "b1", "b2")})
     r = P.check_sampled(w, g, dev, n_tokens=48)
     assert r.route.n_hot_cold.tolist() == [8, 0]
+
+
+def test_large_batch_routing_and_permutation_are_bit_exact():
+    # 40000 assignments: the two-level recount of the permutation (super-chunks of 2048) is exercised,
+    # including a ragged last super-chunk and a ragged last 16-row chunk
+    w = _wl("big_batch", T=20000, d_model=128, d_ff=128, E=48, top_k=2, renormalize=1, hot_threshold=500,
+            zipf_alpha=1.1, bias="none")
+    g = S.generate(w)
+    dev = P.to_device(g)
+    buf = P.run_gpu(w.problem, dev, want_probs=False)
+    P.check_routing(w.problem, g, buf)
