@@ -137,7 +137,9 @@ int monde_permute(const monde_problem* p, const void* x, const int32_t* topk_idx
  *   for e with counts[e] > 0, rows r in [offsets[e], offsets[e+1]):
  *     h[r,:]      = act(x_perm[r,:] * W1[e]^T + b1[e])     (fp32 accumulate, stored in dtype)
  *     y_perm[r,:] = h[r,:] * W2[e]^T + b2[e]               (fp32 accumulate, stored in dtype)
- * Reads counts / offsets / class lists from device memory; nothing comes back to the host.
+ * Reads counts / offsets / classes from device memory; nothing comes back to the host.  cls, hot_ids,
+ * cold_ids and n_hot_cold must describe the same classification (as monde_route and
+ * monde_classify_top_h write them): a kernel may use either form.
  * in : x_perm [A,d_model]; W1 [E,d_ff,d_model]; b1 [E,d_ff] or NULL; W2 [E,d_model,d_ff];
  *      b2 [E,d_model] or NULL (all dtype); counts, offsets, cls, hot_ids, cold_ids,
  *      n_hot_cold as written by monde_route

@@ -148,7 +148,8 @@ int monde_moe_ffn_fwd(const monde_problem* p, const void* x_perm,
         }
         return MONDE_OK;
     }
-    return launch_ffn_bf16(*p, x_perm, W1, b1, W2, b2, counts, offsets, hot_ids, cold_ids, n_hot_cold, y_perm, ws, s);
+    // (the tensor-core kernel rebuilds the class lists from cls, counts and offsets in one pass)
+    return launch_ffn_bf16(*p, x_perm, W1, b1, W2, b2, counts, offsets, cls, y_perm, ws, s);
 }
 
 int monde_combine(const monde_problem* p, const void* y_perm, const int32_t* inv_perm,

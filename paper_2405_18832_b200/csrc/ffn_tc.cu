@@ -77,7 +77,7 @@ enum WaitSite { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3,
                 kSiteHiddenReady = 5, kSiteDrain = 6, kSiteQueue = 7, kSitePartials = 8 };
 
 struct FfnParams {
-    int d_model, d_ff, act;
+    int E, d_model, d_ff, act;
     int cold_tile;                // token tile of the cold class
     int pair_mask;                // bit (class * 2 + layer): units of that segment take two feature tiles
     int n_split;                  // K-splits of a cold second-layer unit (1 = none)
@@ -86,11 +86,9 @@ struct FfnParams {
     const __nv_bfloat16* b2;
     __nv_bfloat16* h;
     __nv_bfloat16* y;
+    const uint8_t* cls;
     const int32_t* counts;
     const int32_t* offsets;
-    const int32_t* hot_ids;
-    const int32_t* cold_ids;
-    const int32_t* n_hot_cold;
     int32_t* status;       // {status, site}
     int32_t* ticket;       // CTAs that have finished
     int32_t* next_unit;    // device-wide unit counter
@@ -344,8 +342,48 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     pdl_wait();
 
     // ---- unit table from the router's outputs -----------------------------------------------
-    ut.n_hot = min(P.n_hot_cold[0], kMaxExperts);
-    ut.n_all = min(ut.n_hot + P.n_hot_cold[1], kMaxExperts);
+    // Thread e reads expert e's class, count and offset (independent loads: one round trip to
+    // memory instead of the three that following n_hot_cold -> id lists -> counts would take) and
+    // the entries are compacted in expert order, which is the order of the router's id lists.
+    __shared__ int s_warp_hot[kThreads / 32], s_warp_cold[kThreads / 32], s_n_hot, s_n_all;
+    {
+        const int e = tid;
+        const int k = e < P.E ? P.cls[e] : 0;
+        const int m = e < P.E ? P.counts[e] : 0;
+        const int off = e < P.E ? P.offsets[e] : 0;
+        const unsigned hot_mask = __ballot_sync(0xffffffffu, k == 2);
+        const unsigned cold_mask = __ballot_sync(0xffffffffu, k == 1);
+        if (lane == 0) {
+            s_warp_hot[warp] = __popc(hot_mask);
+            s_warp_cold[warp] = __popc(cold_mask);
+        }
+        __syncthreads();
+        int hot_before = 0, cold_before = 0, n_hot = 0, n_cold = 0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) {
+            if (w < warp) { hot_before += s_warp_hot[w]; cold_before += s_warp_cold[w]; }
+            n_hot += s_warp_hot[w];
+            n_cold += s_warp_cold[w];
+        }
+        if (tid == 0) { s_n_hot = n_hot; s_n_all = n_hot + n_cold; }
+        if (k != 0) {
+            const bool cold = k == 1;
+            const unsigned lt = (1u << lane) - 1u;
+            const int i = cold ? n_hot + cold_before + __popc(cold_mask & lt) : hot_before + __popc(hot_mask & lt);
+            const int tile = cold ? P.cold_tile : kHotTokTile;
+            const int tt = max(1, (m + tile - 1) / tile);
+            ut.e[i] = e;
+            ut.off[i] = off;
+            ut.m[i] = m;
+            ut.tt[i] = tt;
+            ut.per[i] = ((m + tt - 1) / tt + 15) & ~15;
+            ut.tt_prefix[i + 1] = tt;
+        }
+    }
+    if (tid == 0) ut.tt_prefix[0] = 0;
+    __syncthreads();
+    ut.n_hot = s_n_hot;
+    ut.n_all = s_n_all;
     ut.nt1 = (P.d_ff + kTileRows - 1) / kTileRows;
     ut.nt2 = (P.d_model + kTileRows - 1) / kTileRows;
 #pragma unroll
@@ -353,21 +391,6 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
         ut.tpu[g] = ((P.pair_mask >> g) & 1) + 1;
         ut.upt[g] = (((g & 1) ? ut.nt2 : ut.nt1) + ut.tpu[g] - 1) / ut.tpu[g];
     }
-    for (int i = tid; i < ut.n_all; i += kThreads) {
-        const bool cold = i >= ut.n_hot;
-        const int e = cold ? P.cold_ids[i - ut.n_hot] : P.hot_ids[i];
-        const int tile = cold ? P.cold_tile : kHotTokTile;
-        const int m = P.counts[e];
-        const int tt = max(1, (m + tile - 1) / tile);
-        ut.e[i] = e;
-        ut.off[i] = P.offsets[e];
-        ut.m[i] = m;
-        ut.tt[i] = tt;
-        ut.per[i] = ((m + tt - 1) / tt + 15) & ~15;
-        ut.tt_prefix[i + 1] = tt;
-    }
-    if (tid == 0) ut.tt_prefix[0] = 0;
-    __syncthreads();
     if (warp == 0) {   // inclusive scan of the per-expert token-tile counts, 8 entries per lane
         int v[8], sum = 0;
 #pragma unroll
@@ -484,12 +507,14 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 mbar_arrive(q_full(slot));          // release: the record is visible to whoever acquires
                 return true;
             };
+            // The first unit of CTA c is unit c (no round trip to the counter before the first load);
+            // the counter hands out the units from gridDim.x on.
             Unit cur, nxt;
-            int u = atomicAdd(P.next_unit, 1);
+            const int u = blockIdx.x;
             cur.id = -1;
             if (u < ut.total_units) cur = ut.decode(u);
             ok = push_unit(0, cur);
-            int u_ahead = cur.id >= 0 ? atomicAdd(P.next_unit, 1) : 0;   // consumed a few K blocks later
+            int u_ahead = cur.id >= 0 ? atomicAdd(P.next_unit, 1) + static_cast<int>(gridDim.x) : 0;   // used a few K blocks later
             for (int it = 0; ok && cur.id >= 0; ++it) {
                 const Unit un = cur;
                 trace_mark(P, it, 0, static_cast<unsigned long long>(un.id));
@@ -517,7 +542,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         nxt.id = -1;
                         if (u_ahead < ut.total_units) {
                             nxt = ut.decode(u_ahead);
-                            u_ahead = atomicAdd(P.next_unit, 1);
+                            u_ahead = atomicAdd(P.next_unit, 1) + static_cast<int>(gridDim.x);
                         }
                         if (!push_unit(it + 1, nxt)) { ok = false; break; }
                         next_ready = true;
@@ -893,8 +918,7 @@ int sm_count() {
 
 int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, const void* b1,
                     const void* W2, const void* b2, const int32_t* counts, const int32_t* offsets,
-                    const int32_t* hot_ids, const int32_t* cold_ids, const int32_t* n_hot_cold,
-                    void* y_perm, void* ws, cudaStream_t s) {
+                    const uint8_t* cls, void* y_perm, void* ws, cudaStream_t s) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -908,6 +932,7 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     char* base = static_cast<char*>(ws);
     const uint64_t A = static_cast<uint64_t>(p.T) * p.top_k;
     FfnParams P;
+    P.E = p.E;
     P.d_model = p.d_model;
     P.d_ff = p.d_ff;
     P.act = p.act;
@@ -915,11 +940,9 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.b2 = static_cast<const __nv_bfloat16*>(b2);
     P.h = reinterpret_cast<__nv_bfloat16*>(base + WsLayout::kHidden);
     P.y = static_cast<__nv_bfloat16*>(y_perm);
+    P.cls = cls;
     P.counts = counts;
     P.offsets = offsets;
-    P.hot_ids = hot_ids;
-    P.cold_ids = cold_ids;
-    P.n_hot_cold = n_hot_cold;
     P.status = reinterpret_cast<int32_t*>(base + WsLayout::kStatus);
     P.ticket = reinterpret_cast<int32_t*>(base + WsLayout::kCounters);
     P.next_unit = P.ticket + 1;
