@@ -766,18 +766,20 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     for (int j = 0; j < 16; ++j)
                         sb[j * kTileRows] = __float2bfloat16_rn(__uint_as_float(v[j]) + bias_v);
                 } else {
-                    float acc[16];                                   // fixed order: split 0, 1, .., own
+                    // all partial tiles are requested before any is used: one trip to L2 per group
+                    // instead of one per split; summed in a fixed order: split 0, 1, 2, own
+                    const float* ps = part + c0 * kTileRows;
+                    const int stride = P.cold_tile * kTileRows;
+                    float p0[16], p1[16], p2[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
-#pragma unroll 1
-                    for (int sp = 0; sp + 1 < un.n_split; ++sp) {
-                        const float* ps = part + (sp * P.cold_tile + c0) * kTileRows;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) acc[j] += __ldcg(ps + j * kTileRows);
+                    for (int j = 0; j < 16; ++j) {
+                        p0[j] = __ldcg(ps + j * kTileRows);
+                        p1[j] = un.n_split > 2 ? __ldcg(ps + stride + j * kTileRows) : 0.0f;
+                        p2[j] = un.n_split > 3 ? __ldcg(ps + 2 * stride + j * kTileRows) : 0.0f;
                     }
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        sb[j * kTileRows] = __float2bfloat16_rn(acc[j] + __uint_as_float(v[j]) + bias_v);
+                        sb[j * kTileRows] = __float2bfloat16_rn(((p0[j] + p1[j]) + p2[j]) + __uint_as_float(v[j]) + bias_v);
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 const __nv_bfloat16* rb = stg + (grp & 1) * (16 * kTileRows);
