@@ -51,6 +51,7 @@ namespace monde {
 
 unsigned long long* g_trace = nullptr;
 int g_trace_slots = 0;
+int g_ffn_pair = -1;     // -1: default choice, 0: single CTAs, 1: CTA pairs
 
 namespace {
 
@@ -66,7 +67,8 @@ constexpr int kQueue = 4;            // unit ids in flight between the producer 
 constexpr int kHotTokTile = 256;
 constexpr int kTilesPerUnit = 2;      // a unit covers two 128-feature tiles that share one token tile
 constexpr int kTileBytes = 192 * 1024;
-constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue;
+constexpr int kMailSlots = 8;        // unit indices in flight from the leader of a CTA pair to the other CTA
+constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue + kMailSlots;
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
 constexpr int kStageOutBytes = 2 * 16 * kTileRows * 2;
 constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kQueue * 64 + kTableInts * 4 + kStageOutBytes + 16;
@@ -144,6 +146,7 @@ struct UnitTable {
     int tpu[4];                      // feature tiles per unit, by segment
     int kblocks1, kblocks2;          // 64-wide K blocks of layer 1 (d_model) and layer 2 (d_ff)
     int n_split, kb_per_split, split_major;
+    int pair;                        // 1: every unit is run by a pair of CTAs, one feature tile each
     int seg1, seg2, seg3, total_units;   // list = [hot L1 | hot L2 | cold L1 | cold L2 (split)]
 
     __device__ __forceinline__ Unit decode(int u) const {
@@ -219,7 +222,7 @@ struct UnitTable {
         r.e = e[lo];
         r.n0 = ntile * kTileRows * tpu[sgm];
         r.tiles = min(tpu[sgm], (r.layer ? nt2 : nt1) - tpu[sgm] * ntile);
-        r.wide = !r.cold && tpu[sgm] == 2;
+        r.wide = !pair && !r.cold && tpu[sgm] == 2;
         const int r_in_e = tok * per[lo];
         r.rows = min(per[lo], m[lo] - r_in_e);
         r.nt = (r.rows + 15) & ~15;
@@ -273,7 +276,7 @@ struct FfnMaps {
     CUtensorMap in[2][3];     // [layer][0: 16 rows, 1: 64 rows, 2: 256 rows]
 };
 
-template <int kAct>
+template <int kAct, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_constant__ FfnMaps M, const FfnParams P) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -304,8 +307,15 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     auto rows_stored = [&](int b) { return bar0 + 8u * (kRingBars + 4 + b); };
     auto q_full = [&](int s) { return bar0 + 8u * (kRingBars + 6 + s); };
     auto q_empty = [&](int s) { return bar0 + 8u * (kRingBars + 6 + kQueue + s); };
+    auto mail_bar = [&](int s) { return bar0 + 8u * (kRingBars + 6 + 2 * kQueue + s); };
+    volatile int* mail = reinterpret_cast<volatile int*>(tmem_slot + 4);   // [kMailSlots]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // K blocks per ring stage.  The MMA issuer spends some 400 cycles per stage on barrier probes
+    // and commits, and the tensor core's queue hides only about as much: a stage must carry at
+    // least eight MMAs to keep the tensor core busy.  Single CTAs issue 8 per K block (two feature
+    // tiles), pairs 4 (one 256-row MMA per 16 columns of K), so pairs stage two K blocks at a time.
+    constexpr int kKps = kPair ? 2 : 1;
 
     // ---- set-up that touches nothing another kernel produced: runs while the preceding
     // kernel of the stream is still finishing --------------------------------------------
@@ -322,13 +332,14 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full(b), 1);      // one commit
-            mbar_init(acc_empty(b), 5);     // 4 epilogue warps + the publisher (keeps it at most one use behind)
+            mbar_init(acc_empty(b), kPair ? 10 : 5);   // 4 epilogue warps + the publisher (keeps it at most one use behind), of each CTA
             mbar_init(rows_stored(b), 4);   // 4 epilogue warps
         }
         for (int s = 0; s < kQueue; ++s) {
             mbar_init(q_full(s), 1);        // producer
             mbar_init(q_empty(s), 7);       // MMA issuer, 4 epilogue warps, publisher, token-tile producer
         }
+        for (int s = 0; s < kMailSlots; ++s) mbar_init(mail_bar(s), 1);   // the pair leader's scheduler
         fence_barrier_init();
         for (int l = 0; l < 2; ++l) {
             prefetch_tensormap(&M.w[l][0]);
@@ -336,8 +347,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             for (int i = 0; i < 3; ++i) prefetch_tensormap(&M.in[l][i]);
         }
     } else if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-        tmem_relinquish();
+        if (kPair) {
+            tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+            tmem_relinquish();
+        }
     }
     pdl_wait();
 
@@ -415,14 +431,22 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (kPair) cluster_sync_all();   // the other CTA's barriers and tensor memory exist from here on
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // CTA pairs: rank within the pair, and the leader's copy of the barrier array (the full and
+    // accumulator-free barriers that the MMA issuer waits on live in the leader only).
+    const uint32_t rank = kPair ? cluster_ctarank() : 0u;
+    const uint32_t bar0_leader = kPair ? map_to_cta(bar0, 0) : bar0;
+    const int n_workers = kPair ? static_cast<int>(gridDim.x) / 2 : static_cast<int>(gridDim.x);
+    const int worker = kPair ? static_cast<int>(blockIdx.x) / 2 : static_cast<int>(blockIdx.x);
     const int tt_all = ut.tt_prefix[ut.n_all];
     const int tt_hot = ut.tt_prefix[ut.n_hot];
     ut.kblocks1 = P.d_model / kBlockK;
     ut.kblocks2 = P.d_ff / kBlockK;
     ut.n_split = P.n_split;
     ut.split_major = P.split_major;
+    ut.pair = kPair;
     ut.kb_per_split = (ut.kblocks2 + P.n_split - 1) / P.n_split;
     ut.seg1 = tt_hot * ut.upt[0];
     ut.seg2 = ut.seg1 + tt_hot * ut.upt[1];
@@ -437,9 +461,9 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     struct Geom { int a_bytes, b_bytes, na, nb, b_base; };
     auto geom_of = [&](int g) {
         Geom r;
-        r.a_bytes = ut.tpu[g] * kABytes;
-        r.b_bytes = ((g & 2) ? P.cold_tile : kHotTokTile) * 128;
-        r.nb = (g & 2) ? kMaxStagesB : 3;
+        r.a_bytes = kPair ? kKps * kABytes : ut.tpu[g] * kABytes;                        // per CTA
+        r.b_bytes = ((g & 2) ? P.cold_tile : kHotTokTile) * (kPair ? kKps * 64 : 128);   // a pair holds half the tokens each
+        r.nb = (g & 2) ? 4 : 3;
         r.na = min(kMaxStagesA, (kTileBytes - r.nb * r.b_bytes) / r.a_bytes);
         r.b_base = r.na * r.a_bytes;
         return r;
@@ -507,14 +531,36 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 mbar_arrive(q_full(slot));          // release: the record is visible to whoever acquires
                 return true;
             };
-            // The first unit of CTA c is unit c (no round trip to the counter before the first load);
-            // the counter hands out the units from gridDim.x on.
+            // The first unit of worker w (a CTA, or a CTA pair) is unit w: no round trip to the counter
+            // before the first load.  The counter hands out the rest.  In a CTA pair the
+            // leader draws from the counter and posts the index into the other CTA's mailbox (a
+            // remote store released by a remote mbarrier arrival).  The other CTA's loads gate the
+            // leader's MMAs, so it is never more than five draws behind and eight slots suffice.
+            int draws = 0;
+            auto draw = [&]() -> int { return atomicAdd(P.next_unit, 1) + n_workers; };
+            auto take_next = [&]() -> int {
+                if (!kPair) return draw();
+                const int slot = draws % kMailSlots;
+                const uint32_t parity = (draws / kMailSlots) & 1;
+                ++draws;
+                if (rank == 0) {
+                    const int idx = draw();
+                    st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(mail) + slot), 1), static_cast<uint32_t>(idx));
+                    mbar_arrive_cluster(map_to_cta(mail_bar(slot), 1));
+                    return idx;
+                }
+                if (!mbar_wait_cluster(mail_bar(slot), parity, abort_flag, kWaitLimitNs)) {
+                    report_timeout(P.status, abort_flag, kSiteQueue);
+                    return 0x7fffffff;
+                }
+                return mail[slot];
+            };
             Unit cur, nxt;
-            const int u = blockIdx.x;
+            const int u = worker;
             cur.id = -1;
             if (u < ut.total_units) cur = ut.decode(u);
             ok = push_unit(0, cur);
-            int u_ahead = cur.id >= 0 ? atomicAdd(P.next_unit, 1) + static_cast<int>(gridDim.x) : 0;   // used a few K blocks later
+            int u_ahead = cur.id >= 0 ? take_next() : 0;   // used a few K blocks later
             for (int it = 0; ok && cur.id >= 0; ++it) {
                 const Unit un = cur;
                 trace_mark(P, it, 0, static_cast<unsigned long long>(un.id));
@@ -536,13 +582,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 const CUtensorMap* mw = &M.w[un.layer][un.tiles - 1];   // both feature tiles in one copy
                 const int N = un.layer ? P.d_model : P.d_ff;
                 bool next_ready = false;
-                for (int kb = un.kb0; kb < un.kb1; ++kb) {
-                    if (!next_ready && (kb - un.kb0 == 2 || kb == un.kb1 - 1)) {
+                for (int kb = un.kb0; kb < un.kb1; kb += kKps) {
+                    if (!next_ready && (kb - un.kb0 == 2 || kb + kKps >= un.kb1)) {
                         // take, decode and publish the next unit while this one's loads are in flight
                         nxt.id = -1;
                         if (u_ahead < ut.total_units) {
                             nxt = ut.decode(u_ahead);
-                            u_ahead = atomicAdd(P.next_unit, 1) + static_cast<int>(gridDim.x);
+                            u_ahead = take_next();
                         }
                         if (!push_unit(it + 1, nxt)) { ok = false; break; }
                         next_ready = true;
@@ -553,10 +599,19 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         break;
                     }
                     if (kb == un.kb0) trace_time(P, it, 1);
-                    const uint32_t full = full_a(stage);
                     const uint32_t a_dst = tiles_u32 + stage * gm.a_bytes;
-                    mbar_arrive_expect_tx(full, un.tiles * kABytes);
-                    tma_load_2d(a_dst, mw, full, kb * kBlockK, un.e * N + un.n0, pol_w);
+                    if (kPair) {
+                        // each CTA streams its own feature tile; the leader's barrier counts both
+                        const int nk = min(kKps, un.kb1 - kb);
+                        if (rank == 0) mbar_arrive_expect_tx(full_a(stage), 2 * nk * kABytes);
+                        for (int j = 0; j < nk; ++j)
+                            tma_load_2d_pair(a_dst + j * kABytes, &M.w[un.layer][0], bar0_leader + 8u * stage,
+                                             (kb + j) * kBlockK, un.e * N + un.n0 + static_cast<int>(rank) * kTileRows, pol_w);
+                    } else {
+                        const uint32_t full = full_a(stage);
+                        mbar_arrive_expect_tx(full, un.tiles * kABytes);
+                        tma_load_2d(a_dst, mw, full, kb * kBlockK, un.e * N + un.n0, pol_w);
+                    }
                     fill_bits ^= 1u << stage;
                     if (++stage == gm.na) stage = 0;
                 }
@@ -593,7 +648,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 if (un.layer == 1) {
                     // the hidden rows of this token tile must be complete (its weights already stream)
                     const int32_t* flag = P.ready + un.ready_idx;
-                    const int ready_target = ut.upt[un.cold * 2];   // first-layer units per token tile
+                    const int ready_target = ut.upt[un.cold * 2] * (kPair ? 2 : 1);   // first-layer units per token tile (x CTAs)
                     if (ld_acquire(flag) < ready_target) {
                         const uint64_t t0 = global_timer_ns();
                         while (ld_acquire(flag) < ready_target) {
@@ -607,22 +662,38 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     }
                     fence_proxy_async_all();
                 }
-                for (int kb = un.kb0; kb < un.kb1; ++kb) {
+                for (int kb = un.kb0; kb < un.kb1; kb += kKps) {
                     if (!mbar_wait(empty_b(stage), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteProducerEmpty);
                         ok = false;
                         break;
                     }
-                    const uint32_t full = full_b(stage);
                     const uint32_t b_dst = tiles_u32 + gm.b_base + stage * gm.b_bytes;
-                    mbar_arrive_expect_tx(full, un.nt * 128);
-                    int j = 0;
-                    for (; un.nt - j >= 256; j += 256)
-                        tma_load_2d(b_dst + j * 128, mi + 2, full, kb * kBlockK, un.row0 + j, pol_x);
-                    for (; un.nt - j >= 64; j += 64)
-                        tma_load_2d(b_dst + j * 128, mi + 1, full, kb * kBlockK, un.row0 + j, pol_x);
-                    for (; un.nt - j >= 16; j += 16)
-                        tma_load_2d(b_dst + j * 128, mi, full, kb * kBlockK, un.row0 + j, pol_x);
+                    if (kPair) {
+                        // this CTA's half of the token rows, in boxes of 128, 32 and 8 rows
+                        const int half = un.nt >> 1, r0 = un.row0 + static_cast<int>(rank) * half;
+                        const uint32_t full = bar0_leader + 8u * (2 * kMaxStagesA + stage);
+                        const int nk = min(kKps, un.kb1 - kb);
+                        if (rank == 0) mbar_arrive_expect_tx(full_b(stage), nk * un.nt * 128);
+                        for (int jk = 0; jk < nk; ++jk) {
+                            const uint32_t dst = b_dst + jk * (gm.b_bytes / kKps);
+                            const int x = (kb + jk) * kBlockK;
+                            int j = 0;
+                            for (; half - j >= 128; j += 128) tma_load_2d_pair(dst + j * 128, mi + 2, full, x, r0 + j, pol_x);
+                            for (; half - j >= 32; j += 32) tma_load_2d_pair(dst + j * 128, mi + 1, full, x, r0 + j, pol_x);
+                            for (; half - j >= 8; j += 8) tma_load_2d_pair(dst + j * 128, mi, full, x, r0 + j, pol_x);
+                        }
+                    } else {
+                        const uint32_t full = full_b(stage);
+                        mbar_arrive_expect_tx(full, un.nt * 128);
+                        int j = 0;
+                        for (; un.nt - j >= 256; j += 256)
+                            tma_load_2d(b_dst + j * 128, mi + 2, full, kb * kBlockK, un.row0 + j, pol_x);
+                        for (; un.nt - j >= 64; j += 64)
+                            tma_load_2d(b_dst + j * 128, mi + 1, full, kb * kBlockK, un.row0 + j, pol_x);
+                        for (; un.nt - j >= 16; j += 16)
+                            tma_load_2d(b_dst + j * 128, mi, full, kb * kBlockK, un.row0 + j, pol_x);
+                    }
                     fill_bits ^= 1u << stage;
                     if (++stage == gm.nb) stage = 0;
                 }
@@ -639,6 +710,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             for (int it = 0; ok; ++it) {
                 const Unit un = pop_unit(it, false);
                 if (un.id < 0) break;
+                if (kPair && rank != 0) continue;    // the leader issues for both CTAs
                 if (un.cold * 2 + un.layer != cls) {
                     const Geom g2 = geom_of(un.cold * 2 + un.layer);
                     if (cls < 0 || !same_geom(g2, gm)) {
@@ -656,8 +728,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     break;
                 }
                 tc_fence_after_sync();
-                const uint32_t idesc = idesc_bf16_m128(un.nt);
-                for (int kb = un.kb0; kb < un.kb1; ++kb) {
+                const uint32_t idesc = kPair ? idesc_bf16_m256(un.nt) : idesc_bf16_m128(un.nt);
+                for (int kb = un.kb0; kb < un.kb1; kb += kKps) {
                     if (!mbar_wait(full_a(sa), (use_a >> sa) & 1u, abort_flag, kWaitLimitNs) ||
                         !mbar_wait(full_b(sb), (use_b >> sb) & 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteMmaFull);
@@ -668,21 +740,39 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     if (kb == un.kb0) trace_time(P, it, 3);
                     const uint32_t a_addr = tiles_u32 + sa * gm.a_bytes;
                     const uint64_t b_desc = smem_desc_sw128(tiles_u32 + gm.b_base + sb * gm.b_bytes);
-                    for (int t = 0; t < un.tiles; ++t) {      // feature tiles share the token tile
-                        const uint64_t a_desc = smem_desc_sw128(a_addr + t * kABytes);
+                    if (kPair) {
+                        // 256-row MMAs: this CTA's feature tile and the other CTA's, each against
+                        // all token rows (half of them staged in either CTA); a stage holds two K blocks
+                        const int nk = min(kKps, un.kb1 - kb);
+                        for (int j = 0; j < nk; ++j) {
+                            const uint64_t a_desc = smem_desc_sw128(a_addr + j * kABytes);
+                            const uint64_t bj_desc = smem_desc_sw128(tiles_u32 + gm.b_base + sb * gm.b_bytes + j * (gm.b_bytes / kKps));
 #pragma unroll
-                        for (int k4 = 0; k4 < kBlockK / 16; ++k4)
-                            umma_bf16(tmem_base + acc_col(un, b, t), a_desc + 2 * k4, b_desc + 2 * k4, idesc,
-                                      (kb != un.kb0) | (k4 != 0));
+                            for (int k4 = 0; k4 < kBlockK / 16; ++k4)
+                                umma_bf16_pair(tmem_base + b * 256, a_desc + 2 * k4, bj_desc + 2 * k4, idesc,
+                                               (kb != un.kb0) | (j != 0) | (k4 != 0));
+                        }
+                        umma_commit_pair(empty_a(sa));   // frees the stage in both CTAs
+                        umma_commit_pair(empty_b(sb));
+                    } else {
+                        for (int t = 0; t < un.tiles; ++t) {      // feature tiles share the token tile
+                            const uint64_t a_desc = smem_desc_sw128(a_addr + t * kABytes);
+#pragma unroll
+                            for (int k4 = 0; k4 < kBlockK / 16; ++k4)
+                                umma_bf16(tmem_base + acc_col(un, b, t), a_desc + 2 * k4, b_desc + 2 * k4, idesc,
+                                          (kb != un.kb0) | (k4 != 0));
+                        }
+                        umma_commit(empty_a(sa));   // both stages reusable once these MMAs finish
+                        umma_commit(empty_b(sb));
                     }
-                    umma_commit(empty_a(sa));   // both stages reusable once these MMAs finish
-                    umma_commit(empty_b(sb));
                     use_a ^= 1u << sa;
                     use_b ^= 1u << sb;
                     if (++sa == gm.na) sa = 0;
                     if (++sb == gm.nb) sb = 0;
                 }
-                if (ok) umma_commit(acc_full(b));   // accumulator complete
+                if (ok) {                           // accumulator complete
+                    if (kPair) umma_commit_pair(acc_full(b)); else umma_commit(acc_full(b));
+                }
                 trace_time(P, it, 4);
             }
         }
@@ -718,7 +808,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 if (lane == 0) {
                     const int32_t* flag = P.part_done + un.tile_idx;
                     const uint64_t t0 = global_timer_ns();
-                    while (ld_acquire(flag) < un.n_split - 1) {
+                    while (ld_acquire(flag) < (un.n_split - 1) * (kPair ? 2 : 1)) {
                         if (*abort_flag != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
                             report_timeout(P.status, abort_flag, kSitePartials);
                             break;   // the sums below are wrong but every access stays in bounds
@@ -729,11 +819,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             }
             int grp = 0;       // running 16-token group count: alternates the two staging buffers
 #pragma unroll 1
-            for (int ft = 0; ft < un.tiles; ++ft) {
+            for (int ft = kPair ? static_cast<int>(rank) : 0; ft < (kPair ? static_cast<int>(rank) + 1 : un.tiles); ++ft) {
             const int n0 = un.n0 + ft * kTileRows;
             const int n = n0 + q * 32 + lane;
             const float bias_v = (bias != nullptr && n < N) ? __bfloat162float(bias[static_cast<int64_t>(un.e) * N + n]) : 0.0f;
-            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc_col(un, b, ft);
+            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (kPair ? b * 256 : acc_col(un, b, ft));
             __nv_bfloat16* out = un.layer ? P.y : P.h;
             const int et = tid - 64;                    // 0..127 within the epilogue warps (warps 2-5)
             const int rd_row = et >> 4, rd_col = (et & 15) * 8;
@@ -812,7 +902,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(acc_empty(b));     // accumulator buffer free
+                if (kPair) mbar_arrive_cluster(bar0_leader + 8u * (kRingBars + 2 + b));   // the leader's MMA issuer waits
+                else mbar_arrive(acc_empty(b));     // accumulator buffer free
                 mbar_arrive(rows_stored(b));   // rows stored (release, CTA scope)
                 if (warp == 2) trace_time(P, it, 6);
             }
@@ -834,7 +925,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 // Only now may this accumulator buffer be reused: the epilogue cannot signal "rows
                 // stored" for the buffer's next use before this thread has seen the current one
                 // (a waiter that falls two phases behind an mbarrier would wait on the wrong phase).
-                mbar_arrive(acc_empty(acc.b));
+                if (kPair) mbar_arrive_cluster(bar0_leader + 8u * (kRingBars + 2 + acc.b));
+                else mbar_arrive(acc_empty(acc.b));
                 if (un.layer == 0) {
                     __threadfence();
                     fence_proxy_async_all();
@@ -850,9 +942,10 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     // ---- teardown --------------------------------------------------------------------
     tc_fence_before_sync();
     __syncthreads();
+    if (kPair) cluster_sync_all();   // neither CTA leaves while the other may still signal its barriers
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, kTmemCols);
+        if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols);
     }
     // The last CTA to finish leaves the counters at zero for the next call.
     if (warp == 2) {
@@ -924,11 +1017,13 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(expert_ffn_kernel<MONDE_ACT_RELU>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(expert_ffn_kernel<MONDE_ACT_GELU_ERF>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        const void* kernels[4] = {
+            reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_RELU, false>),
+            reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_GELU_ERF, false>),
+            reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_RELU, true>),
+            reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_GELU_ERF, true>)};
+        for (int i = 0; i < 4 && attr_err == cudaSuccess; ++i)
+            attr_err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     });
     if (attr_err != cudaSuccess) return MONDE_ERR_CUDA;
     char* base = static_cast<char*>(ws);
@@ -955,6 +1050,16 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     // (measured: pairing the hot class takes NLLB-sized layers from 1.53 to 1.39 ms and
     // Switch-Base-sized ones from 175 to 195 us).
     P.pair_mask = 0xC | (p.d_model >= 1536 ? 0x3 : 0);
+    // CTA pairs (one 256-row MMA per pair of SMs, each CTA staging its own feature tile and half of
+    // the token tile) give the hot class the halved token-tile traffic of two-tile units without
+    // filling all of tensor memory, so the epilogue overlaps the next unit's MMAs.  Measured, the
+    // two modes are within 3 % of each other on every workload tried (the feed from L2, about
+    // 11 TB/s over all SMs, limits both), so single CTAs stay the default and pairs are opt-in:
+    // MONDE_FFN_PAIR=1 in the environment, or the internal switch below.
+    static const int pair_env = [] { const char* e = getenv("MONDE_FFN_PAIR"); return e ? atoi(e) : -1; }();
+    const int pair_choice = g_ffn_pair >= 0 ? g_ffn_pair : pair_env;
+    const bool pair = pair_choice > 0;
+    if (pair) P.pair_mask = 0xF;
     const WsLayout L = ws_layout(p);
     P.n_split = L.n_split;
     // Finishing sub-units at the very end of the list give the shortest tail (Switch-Base-sized
@@ -968,7 +1073,8 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.trace = g_trace;
     P.trace_slots = g_trace_slots;
     FfnMaps M;
-    const uint32_t in_box[3] = {16, 64, 256};
+    const uint32_t in_box_single[3] = {16, 64, 256}, in_box_pair[3] = {8, 32, 128};
+    const uint32_t* in_box = pair ? in_box_pair : in_box_single;
     for (int i = 0; i < 2; ++i) {
         if (!make_map(&M.w[0][i], W1, static_cast<uint64_t>(p.E) * p.d_ff, p.d_model, kTileRows << i)) return MONDE_ERR_CUDA;
         if (!make_map(&M.w[1][i], W2, static_cast<uint64_t>(p.E) * p.d_model, p.d_ff, kTileRows << i)) return MONDE_ERR_CUDA;
@@ -978,10 +1084,15 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
         if (!make_map(&M.in[1][i], P.h, A, p.d_ff, in_box[i])) return MONDE_ERR_CUDA;
     }
     cudaError_t err;
-    if (p.act == MONDE_ACT_RELU)
-        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_RELU>, dim3(sm_count()), dim3(kThreads), kSmemBytes, s, M, P);
+    const dim3 grid(pair ? sm_count() & ~1 : sm_count());
+    if (pair && p.act == MONDE_ACT_RELU)
+        err = launch_pdl_cluster(expert_ffn_kernel<MONDE_ACT_RELU, true>, grid, dim3(kThreads), kSmemBytes, 2, s, M, P);
+    else if (pair)
+        err = launch_pdl_cluster(expert_ffn_kernel<MONDE_ACT_GELU_ERF, true>, grid, dim3(kThreads), kSmemBytes, 2, s, M, P);
+    else if (p.act == MONDE_ACT_RELU)
+        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_RELU, false>, grid, dim3(kThreads), kSmemBytes, s, M, P);
     else
-        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_GELU_ERF>, dim3(sm_count()), dim3(kThreads), kSmemBytes, s, M, P);
+        err = launch_pdl(expert_ffn_kernel<MONDE_ACT_GELU_ERF, false>, grid, dim3(kThreads), kSmemBytes, s, M, P);
     if (err != cudaSuccess) return MONDE_ERR_CUDA;
     return launched();
 }
@@ -990,6 +1101,10 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
 
 // Diagnostic hook (not part of the public header): device buffer of 148 * slots * 8 uint64
 // that the FFN kernel fills with a per-unit timeline; pass null to switch it off.
+// Diagnostic / test hook (not part of the public header): 1 runs the expert FFN on CTA pairs
+// (tcgen05 cta_group::2), 0 on single CTAs, -1 restores the default.
+extern "C" void monde_internal_set_ffn_pair(int mode) { monde::g_ffn_pair = mode; }
+
 extern "C" void monde_internal_set_trace(void* device_buf, int slots) {
     monde::g_trace = static_cast<unsigned long long*>(device_buf);
     monde::g_trace_slots = slots;

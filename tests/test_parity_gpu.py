@@ -47,6 +47,29 @@ def test_small_and_edge_cases_match_the_oracle_elementwise(w):
     P.check_full(w)
 
 
+@pytest.fixture
+def cta_pairs():
+    """Runs the expert FFN on CTA pairs (tcgen05 cta_group::2) instead of single CTAs."""
+    B.lib().monde_internal_set_ffn_pair(1)
+    yield
+    B.lib().monde_internal_set_ffn_pair(-1)
+
+
+PAIR_CASES = [w for w in SMALL if w.problem.dtype == "bf16" and w.name in (
+    "bf16_top2_renorm_gelu", "bf16_ragged_tiles", "bf16_all_hot", "bf16_all_cold", "bf16_one_token", "bf16_E256_top8")]
+
+
+@pytest.mark.parametrize("w", PAIR_CASES, ids=[w.name for w in PAIR_CASES])
+def test_cta_pair_mode_matches_the_oracle_elementwise(w, cta_pairs):
+    # odd feature-tile counts (192 = 1.5 tiles, 832 = 6.5), ragged token tiles, split-K cold tiles
+    P.check_full(w)
+
+
+def test_cta_pair_mode_switch_base_like_layer_full_parity(cta_pairs):
+    r = P.check_full(S.config("C1"))
+    assert r.out_err[1] < 4e-3
+
+
 def test_switch_base_like_layer_full_parity():
     r = P.check_full(S.config("C1"))
     assert r.route.n_hot_cold[0] >= 5 and r.route.n_hot_cold[1] >= 40
