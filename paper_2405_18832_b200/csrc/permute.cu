@@ -68,7 +68,31 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
     if (super_before != nullptr)
         for (int e = tid; e < E; e += kThreads) before[e] = super_before[static_cast<size_t>(first / kSuper) * E + e];
     __syncthreads();
-    for (int a = recount_from + tid; a < first; a += kThreads) atomicAdd(&before[topk_idx[a]], 1);
+    // Recount: the loads are batched (four 16-byte loads per thread in flight, 2048 assignments per
+    // trip to L2) because the last chunks look back over thousands of assignments and a load per
+    // loop iteration made them the critical path of the whole call.
+    if ((reinterpret_cast<uintptr_t>(topk_idx) & 15) == 0) {
+        const int4* src4 = reinterpret_cast<const int4*>(topk_idx + recount_from);   // both multiples of 16
+        const int n4 = (first - recount_from) >> 2;
+        for (int i = tid; i < n4; i += 4 * kThreads) {
+            int4 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int q = i + j * kThreads;
+                v[j] = q < n4 ? __ldg(src4 + q) : make_int4(-1, -1, -1, -1);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (v[j].x < 0) continue;
+                atomicAdd(&before[v[j].x], 1);
+                atomicAdd(&before[v[j].y], 1);
+                atomicAdd(&before[v[j].z], 1);
+                atomicAdd(&before[v[j].w], 1);
+            }
+        }
+    } else {
+        for (int a = recount_from + tid; a < first; a += kThreads) atomicAdd(&before[topk_idx[a]], 1);
+    }
     __syncthreads();
     if (warp == 0) {
         const int a = first + lane;

@@ -103,7 +103,28 @@ struct HistArgs {
 __device__ void histogram_classify_scan(const HistArgs& h, const int32_t* __restrict__ topk_idx, int* hist) {
     for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) hist[e] = 0;
     __syncthreads();
-    for (int a = threadIdx.x; a < h.A; a += blockDim.x) atomicAdd(&hist[__ldcg(topk_idx + a)], 1);
+    // The loads are batched (four 16-byte loads per thread in flight): this runs in the last CTA
+    // alone, after everything else, and one load per loop iteration would put A / blockDim.x trips
+    // to L2 on the critical path of the call.
+    const int A4 = (reinterpret_cast<uintptr_t>(topk_idx) & 15) == 0 ? h.A >> 2 : 0;
+    const int4* idx4 = reinterpret_cast<const int4*>(topk_idx);
+    for (int i = threadIdx.x; i < A4; i += 4 * blockDim.x) {
+        int4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int q = i + j * blockDim.x;
+            v[j] = q < A4 ? __ldcg(idx4 + q) : make_int4(-1, -1, -1, -1);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (v[j].x < 0) continue;
+            atomicAdd(&hist[v[j].x], 1);
+            atomicAdd(&hist[v[j].y], 1);
+            atomicAdd(&hist[v[j].z], 1);
+            atomicAdd(&hist[v[j].w], 1);
+        }
+    }
+    for (int a = A4 * 4 + threadIdx.x; a < h.A; a += blockDim.x) atomicAdd(&hist[__ldcg(topk_idx + a)], 1);
     __syncthreads();
     if (threadIdx.x >= 32) return;
     const int lane = threadIdx.x;
