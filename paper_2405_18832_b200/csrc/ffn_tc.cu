@@ -579,11 +579,16 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     }
                     cls = un.cold * 2 + un.layer;
                 }
-                const CUtensorMap* mw = &M.w[un.layer][un.tiles - 1];   // both feature tiles in one copy
+                const CUtensorMap* mw = &M.w[un.layer][kPair ? 0 : un.tiles - 1];   // single CTA: both feature tiles in one copy
                 const int N = un.layer ? P.d_model : P.d_ff;
+                // loop state in registers (see the MMA issuer)
+                const int kb0 = un.kb0, kb1 = un.kb1, a_bytes = gm.a_bytes, na = gm.na;
+                const int w_row = un.e * N + un.n0 + (kPair ? static_cast<int>(rank) * kTileRows : 0);
+                const uint32_t tx_bytes = un.tiles * kABytes;
+                const bool trace_on = P.trace != nullptr;
                 bool next_ready = false;
-                for (int kb = un.kb0; kb < un.kb1; kb += kKps) {
-                    if (!next_ready && (kb - un.kb0 == 2 || kb + kKps >= un.kb1)) {
+                for (int kb = kb0; kb < kb1; kb += kKps) {
+                    if (!next_ready && (kb - kb0 == 2 || kb + kKps >= kb1)) {
                         // take, decode and publish the next unit while this one's loads are in flight
                         nxt.id = -1;
                         if (u_ahead < ut.total_units) {
@@ -598,22 +603,21 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         ok = false;
                         break;
                     }
-                    if (kb == un.kb0) trace_time(P, it, 1);
-                    const uint32_t a_dst = tiles_u32 + stage * gm.a_bytes;
+                    if (trace_on && kb == kb0) trace_time(P, it, 1);
+                    const uint32_t a_dst = tiles_u32 + stage * a_bytes;
                     if (kPair) {
                         // each CTA streams its own feature tile; the leader's barrier counts both
-                        const int nk = min(kKps, un.kb1 - kb);
+                        const int nk = min(kKps, kb1 - kb);
                         if (rank == 0) mbar_arrive_expect_tx(full_a(stage), 2 * nk * kABytes);
                         for (int j = 0; j < nk; ++j)
-                            tma_load_2d_pair(a_dst + j * kABytes, &M.w[un.layer][0], bar0_leader + 8u * stage,
-                                             (kb + j) * kBlockK, un.e * N + un.n0 + static_cast<int>(rank) * kTileRows, pol_w);
+                            tma_load_2d_pair(a_dst + j * kABytes, mw, bar0_leader + 8u * stage, (kb + j) * kBlockK, w_row, pol_w);
                     } else {
                         const uint32_t full = full_a(stage);
-                        mbar_arrive_expect_tx(full, un.tiles * kABytes);
-                        tma_load_2d(a_dst, mw, full, kb * kBlockK, un.e * N + un.n0, pol_w);
+                        mbar_arrive_expect_tx(full, tx_bytes);
+                        tma_load_2d(a_dst, mw, full, kb * kBlockK, w_row, pol_w);
                     }
                     fill_bits ^= 1u << stage;
-                    if (++stage == gm.na) stage = 0;
+                    if (++stage == na) stage = 0;
                 }
                 trace_time(P, it, 2);
                 cur = nxt;
@@ -662,21 +666,24 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     }
                     fence_proxy_async_all();
                 }
-                for (int kb = un.kb0; kb < un.kb1; kb += kKps) {
+                // loop state in registers (see the MMA issuer)
+                const int kb0 = un.kb0, kb1 = un.kb1, nt = un.nt, row0 = un.row0, b_bytes = gm.b_bytes, nb = gm.nb;
+                const uint32_t b_ring = tiles_u32 + gm.b_base;
+                for (int kb = kb0; kb < kb1; kb += kKps) {
                     if (!mbar_wait(empty_b(stage), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteProducerEmpty);
                         ok = false;
                         break;
                     }
-                    const uint32_t b_dst = tiles_u32 + gm.b_base + stage * gm.b_bytes;
+                    const uint32_t b_dst = b_ring + stage * b_bytes;
                     if (kPair) {
                         // this CTA's half of the token rows, in boxes of 128, 32 and 8 rows
-                        const int half = un.nt >> 1, r0 = un.row0 + static_cast<int>(rank) * half;
+                        const int half = nt >> 1, r0 = row0 + static_cast<int>(rank) * half;
                         const uint32_t full = bar0_leader + 8u * (2 * kMaxStagesA + stage);
-                        const int nk = min(kKps, un.kb1 - kb);
-                        if (rank == 0) mbar_arrive_expect_tx(full_b(stage), nk * un.nt * 128);
+                        const int nk = min(kKps, kb1 - kb);
+                        if (rank == 0) mbar_arrive_expect_tx(full_b(stage), nk * nt * 128);
                         for (int jk = 0; jk < nk; ++jk) {
-                            const uint32_t dst = b_dst + jk * (gm.b_bytes / kKps);
+                            const uint32_t dst = b_dst + jk * (b_bytes / kKps);
                             const int x = (kb + jk) * kBlockK;
                             int j = 0;
                             for (; half - j >= 128; j += 128) tma_load_2d_pair(dst + j * 128, mi + 2, full, x, r0 + j, pol_x);
@@ -685,17 +692,17 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         }
                     } else {
                         const uint32_t full = full_b(stage);
-                        mbar_arrive_expect_tx(full, un.nt * 128);
+                        mbar_arrive_expect_tx(full, nt * 128);
                         int j = 0;
-                        for (; un.nt - j >= 256; j += 256)
-                            tma_load_2d(b_dst + j * 128, mi + 2, full, kb * kBlockK, un.row0 + j, pol_x);
-                        for (; un.nt - j >= 64; j += 64)
-                            tma_load_2d(b_dst + j * 128, mi + 1, full, kb * kBlockK, un.row0 + j, pol_x);
-                        for (; un.nt - j >= 16; j += 16)
-                            tma_load_2d(b_dst + j * 128, mi, full, kb * kBlockK, un.row0 + j, pol_x);
+                        for (; nt - j >= 256; j += 256)
+                            tma_load_2d(b_dst + j * 128, mi + 2, full, kb * kBlockK, row0 + j, pol_x);
+                        for (; nt - j >= 64; j += 64)
+                            tma_load_2d(b_dst + j * 128, mi + 1, full, kb * kBlockK, row0 + j, pol_x);
+                        for (; nt - j >= 16; j += 16)
+                            tma_load_2d(b_dst + j * 128, mi, full, kb * kBlockK, row0 + j, pol_x);
                     }
                     fill_bits ^= 1u << stage;
-                    if (++stage == gm.nb) stage = 0;
+                    if (++stage == nb) stage = 0;
                 }
             }
         }
@@ -729,7 +736,16 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 }
                 tc_fence_after_sync();
                 const uint32_t idesc = kPair ? idesc_bf16_m256(un.nt) : idesc_bf16_m128(un.nt);
-                for (int kb = un.kb0; kb < un.kb1; kb += kKps) {
+                // Everything the K loop needs sits in registers: this thread's instruction stream is
+                // what feeds the tensor core, and a reload after every inline-assembly statement
+                // (they act as compiler barriers) showed up as hundreds of cycles per K block.
+                const int kb0 = un.kb0, kb1 = un.kb1, tiles = un.tiles;
+                const int a_bytes = gm.a_bytes, b_bytes = gm.b_bytes, na = gm.na, nb = gm.nb;
+                const uint32_t a_ring = tiles_u32, b_ring = tiles_u32 + gm.b_base;
+                const uint32_t acc0 = tmem_base + (kPair ? b * 256 : acc_col(un, b, 0));
+                const uint32_t acc1 = tmem_base + (kPair ? b * 256 : acc_col(un, b, 1));
+                const bool trace_on = P.trace != nullptr;
+                for (int kb = kb0; kb < kb1; kb += kKps) {
                     if (!mbar_wait(full_a(sa), (use_a >> sa) & 1u, abort_flag, kWaitLimitNs) ||
                         !mbar_wait(full_b(sb), (use_b >> sb) & 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteMmaFull);
@@ -737,38 +753,42 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         break;
                     }
                     tc_fence_after_sync();
-                    if (kb == un.kb0) trace_time(P, it, 3);
-                    const uint32_t a_addr = tiles_u32 + sa * gm.a_bytes;
-                    const uint64_t b_desc = smem_desc_sw128(tiles_u32 + gm.b_base + sb * gm.b_bytes);
+                    if (trace_on && kb == kb0) trace_time(P, it, 3);
+                    const uint32_t a_addr = a_ring + sa * a_bytes;
+                    const uint32_t b_addr = b_ring + sb * b_bytes;
+                    const uint32_t later = kb != kb0;      // 0 for the K block that initialises the accumulator
                     if (kPair) {
                         // 256-row MMAs: this CTA's feature tile and the other CTA's, each against
                         // all token rows (half of them staged in either CTA); a stage holds two K blocks
-                        const int nk = min(kKps, un.kb1 - kb);
+                        const int nk = min(kKps, kb1 - kb);
                         for (int j = 0; j < nk; ++j) {
                             const uint64_t a_desc = smem_desc_sw128(a_addr + j * kABytes);
-                            const uint64_t bj_desc = smem_desc_sw128(tiles_u32 + gm.b_base + sb * gm.b_bytes + j * (gm.b_bytes / kKps));
+                            const uint64_t bj_desc = smem_desc_sw128(b_addr + j * (b_bytes / kKps));
 #pragma unroll
                             for (int k4 = 0; k4 < kBlockK / 16; ++k4)
-                                umma_bf16_pair(tmem_base + b * 256, a_desc + 2 * k4, bj_desc + 2 * k4, idesc,
-                                               (kb != un.kb0) | (j != 0) | (k4 != 0));
+                                umma_bf16_pair(acc0, a_desc + 2 * k4, bj_desc + 2 * k4, idesc, later | (j != 0) | (k4 != 0));
                         }
                         umma_commit_pair(empty_a(sa));   // frees the stage in both CTAs
                         umma_commit_pair(empty_b(sb));
                     } else {
-                        for (int t = 0; t < un.tiles; ++t) {      // feature tiles share the token tile
-                            const uint64_t a_desc = smem_desc_sw128(a_addr + t * kABytes);
+                        const uint64_t b_desc = smem_desc_sw128(b_addr);
+                        const uint64_t a_desc = smem_desc_sw128(a_addr);
+#pragma unroll
+                        for (int k4 = 0; k4 < kBlockK / 16; ++k4)
+                            umma_bf16(acc0, a_desc + 2 * k4, b_desc + 2 * k4, idesc, later | (k4 != 0));
+                        if (tiles == 2) {                  // the second feature tile shares the token tile
+                            const uint64_t a1_desc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
                             for (int k4 = 0; k4 < kBlockK / 16; ++k4)
-                                umma_bf16(tmem_base + acc_col(un, b, t), a_desc + 2 * k4, b_desc + 2 * k4, idesc,
-                                          (kb != un.kb0) | (k4 != 0));
+                                umma_bf16(acc1, a1_desc + 2 * k4, b_desc + 2 * k4, idesc, later | (k4 != 0));
                         }
                         umma_commit(empty_a(sa));   // both stages reusable once these MMAs finish
                         umma_commit(empty_b(sb));
                     }
                     use_a ^= 1u << sa;
                     use_b ^= 1u << sb;
-                    if (++sa == gm.na) sa = 0;
-                    if (++sb == gm.nb) sb = 0;
+                    if (++sa == na) sa = 0;
+                    if (++sb == nb) sb = 0;
                 }
                 if (ok) {                           // accumulator complete
                     if (kPair) umma_commit_pair(acc_full(b)); else umma_commit(acc_full(b));
@@ -802,13 +822,15 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             if (warp == 2 && lane == 0) trace_time(P, it, 5);
             const int N = un.layer ? P.d_model : P.d_ff;
             const __nv_bfloat16* bias = un.layer ? P.b2 : P.b1;
-            const bool is_partial = un.split + 1 < un.n_split;
-            if (un.n_split > 1 && !is_partial) {
+            // unit fields used per token group, in registers (see the MMA issuer)
+            const int u_rows = un.rows, u_row0 = un.row0, u_nt = un.nt, u_split = un.split, u_nsplit = un.n_split;
+            const bool is_partial = u_split + 1 < u_nsplit;
+            if (u_nsplit > 1 && !is_partial) {
                 // finishing sub-unit: the partial tiles were taken from the list before this one
                 if (lane == 0) {
                     const int32_t* flag = P.part_done + un.tile_idx;
                     const uint64_t t0 = global_timer_ns();
-                    while (ld_acquire(flag) < (un.n_split - 1) * (kPair ? 2 : 1)) {
+                    while (ld_acquire(flag) < (u_nsplit - 1) * (kPair ? 2 : 1)) {
                         if (*abort_flag != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
                             report_timeout(P.status, abort_flag, kSitePartials);
                             break;   // the sums below are wrong but every access stays in bounds
@@ -834,16 +856,17 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             // instruction cache and ran 20x slower.
             // K-split tiles: fp32 partials live as [split][token][feature] so that a warp touches
             // 128 contiguous bytes per token.
-            float* part = P.partials + static_cast<size_t>(un.tile_idx * kTilesPerUnit + ft) * (un.n_split - 1) *
-                                           (P.cold_tile * kTileRows) + q * 32 + lane;
+            const int cold_tile = P.cold_tile;
+            float* part = P.partials + static_cast<size_t>(un.tile_idx * kTilesPerUnit + ft) * (u_nsplit - 1) *
+                                           (cold_tile * kTileRows) + q * 32 + lane;
             // One group = 16 tokens.  mode: 0 first layer (activation), 1 second layer, 2 second
             // layer finishing a K-split tile (adds the partial tiles), 3 partial tile (fp32 store).
-            const int mode = un.layer == 0 ? 0 : (un.n_split == 1 ? 1 : (is_partial ? 3 : 2));
+            const int mode = un.layer == 0 ? 0 : (u_nsplit == 1 ? 1 : (is_partial ? 3 : 2));
             auto drain16 = [&](const uint32_t (&v)[16], int c0) {
                 if (mode == 3) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        part[(un.split * P.cold_tile + c0 + j) * kTileRows] = __uint_as_float(v[j]);
+                        part[(u_split * cold_tile + c0 + j) * kTileRows] = __uint_as_float(v[j]);
                     return;
                 }
                 __nv_bfloat16* sb = stg + (grp & 1) * (16 * kTileRows) + q * 32 + lane;
@@ -859,13 +882,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     // all partial tiles are requested before any is used: one trip to L2 per group
                     // instead of one per split; summed in a fixed order: split 0, 1, 2, own
                     const float* ps = part + c0 * kTileRows;
-                    const int stride = P.cold_tile * kTileRows;
+                    const int stride = cold_tile * kTileRows;
                     float p0[16], p1[16], p2[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         p0[j] = __ldcg(ps + j * kTileRows);
-                        p1[j] = un.n_split > 2 ? __ldcg(ps + stride + j * kTileRows) : 0.0f;
-                        p2[j] = un.n_split > 3 ? __ldcg(ps + 2 * stride + j * kTileRows) : 0.0f;
+                        p1[j] = u_nsplit > 2 ? __ldcg(ps + stride + j * kTileRows) : 0.0f;
+                        p2[j] = u_nsplit > 3 ? __ldcg(ps + 2 * stride + j * kTileRows) : 0.0f;
                     }
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
@@ -877,9 +900,9 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     const int r = rd_row + half * 8;
-                    if (col_ok && c0 + r < un.rows) {
+                    if (col_ok && c0 + r < u_rows) {
                         const uint4 val = *reinterpret_cast<const uint4*>(rb + r * kTileRows + rd_col);
-                        *reinterpret_cast<uint4*>(out + static_cast<int64_t>(un.row0 + c0 + r) * N + n0 + rd_col) = val;
+                        *reinterpret_cast<uint4*>(out + static_cast<int64_t>(u_row0 + c0 + r) * N + n0 + rd_col) = val;
                     }
                 }
             };
@@ -888,13 +911,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             uint32_t va[16], vb[16];
             tmem_ld_16(t_addr, va);
 #pragma unroll 1
-            for (int c0 = 0; c0 < un.nt; c0 += 32) {
+            for (int c0 = 0; c0 < u_nt; c0 += 32) {
                 tmem_ld_wait();
-                if (c0 + 16 < un.nt) tmem_ld_16(t_addr + c0 + 16, vb);
+                if (c0 + 16 < u_nt) tmem_ld_16(t_addr + c0 + 16, vb);
                 drain16(va, c0);
-                if (c0 + 16 < un.nt) {
+                if (c0 + 16 < u_nt) {
                     tmem_ld_wait();
-                    if (c0 + 32 < un.nt) tmem_ld_16(t_addr + c0 + 32, va);
+                    if (c0 + 32 < u_nt) tmem_ld_16(t_addr + c0 + 32, va);
                     drain16(vb, c0 + 16);
                 }
             }
