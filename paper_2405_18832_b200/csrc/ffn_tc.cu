@@ -745,9 +745,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 const uint32_t acc0 = tmem_base + (kPair ? b * 256 : acc_col(un, b, 0));
                 const uint32_t acc1 = tmem_base + (kPair ? b * 256 : acc_col(un, b, 1));
                 const bool trace_on = P.trace != nullptr;
+                bool stage_ready = false;       // the next K block's barriers were probed during this one's MMAs
                 for (int kb = kb0; kb < kb1; kb += kKps) {
-                    if (!mbar_wait(full_a(sa), (use_a >> sa) & 1u, abort_flag, kWaitLimitNs) ||
-                        !mbar_wait(full_b(sb), (use_b >> sb) & 1u, abort_flag, kWaitLimitNs)) {
+                    if (!stage_ready &&
+                        (!mbar_wait(full_a(sa), (use_a >> sa) & 1u, abort_flag, kWaitLimitNs) ||
+                         !mbar_wait(full_b(sb), (use_b >> sb) & 1u, abort_flag, kWaitLimitNs))) {
                         report_timeout(P.status, abort_flag, kSiteMmaFull);
                         ok = false;
                         break;
@@ -773,9 +775,12 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     } else {
                         const uint64_t b_desc = smem_desc_sw128(b_addr);
                         const uint64_t a_desc = smem_desc_sw128(a_addr);
-#pragma unroll
-                        for (int k4 = 0; k4 < kBlockK / 16; ++k4)
-                            umma_bf16(acc0, a_desc + 2 * k4, b_desc + 2 * k4, idesc, later | (k4 != 0));
+                        // rings have at least three stages, so the next stage is not this one and its use
+                        // bit is still that of its next fill; past the unit's last K block the answer is unused
+                        const int sa_next = sa + 1 == na ? 0 : sa + 1, sb_next = sb + 1 == nb ? 0 : sb + 1;
+                        stage_ready = umma_bf16_x4_probe(acc0, a_desc, b_desc, idesc, later, full_a(sa_next),
+                                                         (use_a >> sa_next) & 1u, full_b(sb_next), (use_b >> sb_next) & 1u) &&
+                                      kb + 1 < kb1;
                         if (tiles == 2) {                  // the second feature tile shares the token tile
                             const uint64_t a1_desc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll

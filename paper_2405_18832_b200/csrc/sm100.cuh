@@ -110,6 +110,36 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) );
 }
+// Four MMAs over one 64-wide K block (descriptors advance by 32 bytes per 16 columns) with a
+// non-blocking probe of two mbarriers issued first and read last: the probes take over a
+// hundred cycles to answer, and the issuing thread would otherwise sit out that time before
+// every K block.  `accumulate` applies to the first MMA; the other three always accumulate.
+// Returns true when both probed phases are complete.
+__device__ __forceinline__ bool umma_bf16_x4_probe(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                   uint32_t accumulate, uint32_t bar_a, uint32_t parity_a,
+                                                   uint32_t bar_b, uint32_t parity_b) {
+    uint32_t ready;
+    asm volatile(
+        "{\n\t.reg .pred pa, pb, p, t;\n\t.reg .b64 a, b;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 pa, [%6], %7;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 pb, [%8], %9;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "setp.eq.b32 t, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t"
+        "add.s64 a, %2, 2;\n\tadd.s64 b, %3, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], a, b, %4, t;\n\t"
+        "add.s64 a, %2, 4;\n\tadd.s64 b, %3, 4;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], a, b, %4, t;\n\t"
+        "add.s64 a, %2, 6;\n\tadd.s64 b, %3, 6;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], a, b, %4, t;\n\t"
+        "and.pred pa, pa, pb;\n\t"
+        "selp.u32 %0, 1, 0, pa;\n\t}"
+        : "=r"(ready)
+        : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(bar_a), "r"(parity_a), "r"(bar_b),
+          "r"(parity_b)
+        : "memory");
+    return ready != 0;
+}
 // Arrives on `bar` once every tcgen05.mma issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
