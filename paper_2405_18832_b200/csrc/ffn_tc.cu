@@ -35,9 +35,10 @@
 // megabyte alone.  Sub-units 0..S-2 store fp32 partial tiles in the workspace; the last
 // sub-unit (again later in the list than the ones it waits for) adds them in a fixed
 // order, so results stay bit-reproducible.
-// Warp roles: warp 0 issues TMA, warp 1 issues MMAs and owns the TMEM allocation, warps
-// 2-5 drain the accumulator (bias + activation fused) while the next unit's MMAs run into
-// the second accumulator buffer.  Counts never travel to the host.
+// Warp roles: warp 0 schedules and issues the weight-tile TMA loads, warp 7 the token-tile
+// loads, warp 1 issues MMAs and owns the TMEM allocation, warps 2-5 and 8-11 drain the
+// accumulator (bias + activation fused) while the next unit's MMAs run into the second
+// accumulator buffer, warp 6 publishes finished rows.  Counts never travel to the host.
 #include <cuda.h>
 
 #include <algorithm>
@@ -57,7 +58,7 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 256;       // weight producer, MMA, 4 epilogue warps, publisher, token-tile producer
+constexpr int kThreads = 384;       // weight producer, MMA, 4 epilogue warps, publisher, token-tile producer, 4 more epilogue warps
 constexpr int kBlockK = 64;           // K elements per stage: one 128-byte swizzle row
 constexpr int kTileRows = 128;        // output features per unit = MMA M
 constexpr int kABytes = kTileRows * 128;
@@ -70,7 +71,7 @@ constexpr int kTileBytes = 192 * 1024;
 constexpr int kMailSlots = 8;        // unit indices in flight from the leader of a CTA pair to the other CTA
 constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue + kMailSlots;
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
-constexpr int kStageOutBytes = 2 * 16 * kTileRows * 2;
+constexpr int kStageOutBytes = 2 * 2 * 16 * kTileRows * 2;   // per epilogue warp set: two staging buffers of 16 tokens x 128 features
 constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kQueue * 64 + kTableInts * 4 + kStageOutBytes + 16;
 constexpr int kTmemCols = 512;        // two accumulator buffers of 256 fp32 columns
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
@@ -285,7 +286,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* unit_queue = reinterpret_cast<int*>(tmem_slot + 16);      // [kQueue] decoded units, 16 ints each
     int* tab = unit_queue + kQueue * 16;
-    __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(                     // 2 x [16 tokens][128 features]
+    __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(                     // 2 sets x 2 x [16 tokens][128 features]
         (reinterpret_cast<uintptr_t>(tab + kTableInts) + 15) & ~uintptr_t(15));
     UnitTable ut;
     ut.tt_prefix = tab;
@@ -332,12 +333,12 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full(b), 1);      // one commit
-            mbar_init(acc_empty(b), kPair ? 10 : 5);   // 4 epilogue warps + the publisher (keeps it at most one use behind), of each CTA
-            mbar_init(rows_stored(b), 4);   // 4 epilogue warps
+            mbar_init(acc_empty(b), kPair ? 18 : 9);   // 8 epilogue warps + the publisher (keeps it at most one use behind), of each CTA
+            mbar_init(rows_stored(b), 8);   // 8 epilogue warps
         }
         for (int s = 0; s < kQueue; ++s) {
             mbar_init(q_full(s), 1);        // producer
-            mbar_init(q_empty(s), 7);       // MMA issuer, 4 epilogue warps, publisher, token-tile producer
+            mbar_init(q_empty(s), 11);      // MMA issuer, 8 epilogue warps, publisher, token-tile producer
         }
         for (int s = 0; s < kMailSlots; ++s) mbar_init(mail_bar(s), 1);   // the pair leader's scheduler
         fence_barrier_init();
@@ -801,9 +802,15 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 trace_time(P, it, 4);
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 6 || warp >= 8) {
         // ---- epilogue: TMEM -> registers -> bias, activation -> shared -> global -------------
+        // Two sets of four warps (2-5 and 8-11): a warp may only read the TMEM lanes of quarter warp % 4,
+        // so each set covers all 128 features; set s drains the 16-token groups of parity s.  One warp per
+        // scheduler did not hide the latencies of its own 110 instructions per group; two interleave.
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int set = warp >= 8;
+        const int bar_id = 1 + set;             // named barrier of the set
+        __nv_bfloat16* const stg_set = stg + set * (2 * 16 * kTileRows);
         AccCursor acc;
         for (int it = 0;; ++it) {
             const Unit un = pop_unit(it, true);
@@ -819,9 +826,9 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             asm volatile(
                 "{\n\t.reg .pred p, q;\n\t"
                 "setp.ne.u32 q, %1, 0;\n\t"
-                "bar.red.and.pred p, 1, 128, q;\n\t"
+                "bar.red.and.pred p, %2, 128, q;\n\t"
                 "selp.u32 %0, 1, 0, p;\n\t}"
-                : "=r"(all_got) : "r"(static_cast<uint32_t>(got)) : "memory");
+                : "=r"(all_got) : "r"(static_cast<uint32_t>(got)), "r"(bar_id) : "memory");
             if (!all_got) break;
             tc_fence_after_sync();
             if (warp == 2 && lane == 0) trace_time(P, it, 5);
@@ -852,7 +859,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             const float bias_v = (bias != nullptr && n < N) ? __bfloat162float(bias[static_cast<int64_t>(un.e) * N + n]) : 0.0f;
             const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (kPair ? b * 256 : acc_col(un, b, ft));
             __nv_bfloat16* out = un.layer ? P.y : P.h;
-            const int et = tid - 64;                    // 0..127 within the epilogue warps (warps 2-5)
+            const int et = set ? tid - 256 : tid - 64;   // 0..127 within the set
             const int rd_row = et >> 4, rd_col = (et & 15) * 8;
             const bool col_ok = n0 + rd_col < N;     // N is a multiple of 64: 8-wide groups are all in or all out
             // Each group of 16 tokens is transposed through shared memory so that global stores are
@@ -874,7 +881,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         part[(u_split * cold_tile + c0 + j) * kTileRows] = __uint_as_float(v[j]);
                     return;
                 }
-                __nv_bfloat16* sb = stg + (grp & 1) * (16 * kTileRows) + q * 32 + lane;
+                __nv_bfloat16* sb = stg_set + (grp & 1) * (16 * kTileRows) + q * 32 + lane;
                 if (mode == 0) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
@@ -899,8 +906,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     for (int j = 0; j < 16; ++j)
                         sb[j * kTileRows] = __float2bfloat16_rn(((p0[j] + p1[j]) + p2[j]) + __uint_as_float(v[j]) + bias_v);
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                const __nv_bfloat16* rb = stg + (grp & 1) * (16 * kTileRows);
+                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+                const __nv_bfloat16* rb = stg_set + (grp & 1) * (16 * kTileRows);
                 ++grp;
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
@@ -914,16 +921,17 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             // Two 16-column loads in flight, ping-pong; the loop is kept rolled so that the whole
             // epilogue stays a few KB of code.
             uint32_t va[16], vb[16];
-            tmem_ld_16(t_addr, va);
+            int c0 = 16 * set;
+            if (c0 < u_nt) tmem_ld_16(t_addr + c0, va);
 #pragma unroll 1
-            for (int c0 = 0; c0 < u_nt; c0 += 32) {
+            for (; c0 < u_nt; c0 += 64) {
                 tmem_ld_wait();
-                if (c0 + 16 < u_nt) tmem_ld_16(t_addr + c0 + 16, vb);
+                if (c0 + 32 < u_nt) tmem_ld_16(t_addr + c0 + 32, vb);
                 drain16(va, c0);
-                if (c0 + 16 < u_nt) {
+                if (c0 + 32 < u_nt) {
                     tmem_ld_wait();
-                    if (c0 + 32 < u_nt) tmem_ld_16(t_addr + c0 + 32, va);
-                    drain16(vb, c0 + 16);
+                    if (c0 + 64 < u_nt) tmem_ld_16(t_addr + c0 + 64, va);
+                    drain16(vb, c0 + 32);
                 }
             }
             }   // feature tiles of the unit
