@@ -214,3 +214,52 @@ def moe_ffn_layer_forward_host(p, x_host, out_host, Wg, bg, W1, b1, W2, b2, buf:
     out_host.copy_(out, non_blocking=True)
     (torch.cuda.current_stream() if stream is None else stream).synchronize()
     return out_host
+
+
+class HostPipeline:
+    """Layer steps whose tokens live in pinned host memory, pipelined over three streams.
+
+    The copy of step n+1's tokens to the device and the copy of step n-1's result back to the
+    host run while step n computes: `depth` sets of device buffers take turns, events order the
+    streams, and the host never waits inside `submit`.  Every step still does its own
+    host->device copy, its four calls and its device->host copy; only their overlap across
+    steps differs from `moe_ffn_layer_forward_host`.
+    """
+
+    def __init__(self, p, depth: int = 2, device="cuda"):
+        self.p = p
+        self.depth = depth
+        self.bufs = [LayerBuffers(p, device=device) for _ in range(depth)]
+        self.s_in = torch.cuda.Stream(device=device)
+        self.s_run = torch.cuda.Stream(device=device)
+        self.s_out = torch.cuda.Stream(device=device)
+        self.copied_in = [torch.cuda.Event() for _ in range(depth)]
+        self.computed = [torch.cuda.Event() for _ in range(depth)]
+        self.copied_out = [torch.cuda.Event() for _ in range(depth)]
+        self.steps = 0
+
+    def submit(self, x_host, out_host, Wg, bg, W1, b1, W2, b2) -> None:
+        """Enqueues one step; `out_host` holds its result once `wait()` (or a later event) says so."""
+        i = self.steps % self.depth
+        buf = self.bufs[i]
+        reused = self.steps >= self.depth
+        if reused:
+            self.s_in.wait_event(self.computed[i])        # the step that last read this x_dev has run
+        with torch.cuda.stream(self.s_in):
+            buf.x_dev.copy_(x_host, non_blocking=True)
+        self.copied_in[i].record(self.s_in)
+        self.s_run.wait_event(self.copied_in[i])
+        if reused:
+            self.s_run.wait_event(self.copied_out[i])     # this buffer set's previous result has left
+        moe_ffn_layer_forward(self.p, buf.x_dev, Wg, bg, W1, b1, W2, b2, buf, self.s_run)
+        self.computed[i].record(self.s_run)
+        self.s_out.wait_event(self.computed[i])
+        with torch.cuda.stream(self.s_out):
+            out_host.copy_(buf.out, non_blocking=True)
+        self.copied_out[i].record(self.s_out)
+        self.steps += 1
+
+    def wait(self) -> None:
+        self.s_out.synchronize()
+        for buf in self.bufs:
+            monde_poll_device_status(buf.ws, self.s_run)
