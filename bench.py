@@ -233,6 +233,8 @@ def run_ours(args, w):
     stream = torch.cuda.current_stream()
     L = B.lib()
 
+    fuse = bool(args.fuse_combine) and p.top_k == 1 and p.dtype == "bf16"
+
     def layer(ev=None):
         if ev is not None:
             ev[0].record(stream)
@@ -246,6 +248,13 @@ def run_ours(args, w):
         B.monde_permute(p, d["x"], buf.topk_idx, buf.offsets, buf.perm, buf.inv_perm, buf.x_perm, buf.ws)
         if ev is not None:
             ev[2].record(stream)
+        if fuse:       # three-call form: the FFN's last store applies the gate weight and writes `out`
+            B.monde_moe_ffn_combine_fwd(p, buf.x_perm, d["W1"], d["b1"], d["W2"], d["b2"], buf.counts, buf.offsets,
+                                        buf.cls, buf.perm, buf.topk_w, buf.out, buf.ws)
+            if ev is not None:
+                ev[3].record(stream)
+                ev[4].record(stream)
+            return
         B.monde_moe_ffn_fwd(p, buf.x_perm, d["W1"], d["b1"], d["W2"], d["b2"], buf.counts, buf.offsets, buf.cls,
                             buf.hot_ids, buf.cold_ids, buf.n_hot_cold, buf.y_perm, buf.ws)
         if ev is not None:
@@ -386,6 +395,7 @@ def run_ours(args, w):
                      "ffn": ffn_ms, "combine": statistics.mean(call_ms[3])},
         "calls_ms_sum": sum(statistics.mean(c) for c in call_ms),
         "layer_hbm_floor_ms": layer_floor_ms, "layer_roofline_frac": layer_floor_ms / ms_per_step,
+        "calls": "route, permute, ffn+combine (fused last store)" if fuse else "route, permute, ffn, combine",
         "policy": args.policy if args.policy == "threshold" else
         f"top_h alpha={args.alpha} bw_hot={args.bw_hot} bw_cold={args.bw_cold}",
         "routing": {"active": int((counts > 0).sum()), "hot": n_hot_used,
@@ -406,6 +416,8 @@ def main():
                     help="C1 (default), C2, C3, or a crossover-sweep point C4:<d_model>:<T>:<zipf alpha>:<threshold>")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fuse-combine", action="store_true",
+                    help="top-1 workloads: monde_moe_ffn_combine_fwd instead of monde_moe_ffn_fwd + monde_combine")
     ap.add_argument("--policy", default="threshold", choices=["threshold", "top_h"],
                     help="hot/cold rule: count >= hot_threshold, or the paper's top-H rule (Eq. 6)")
     ap.add_argument("--alpha", type=float, default=1.0, help="Eq. 6 tuning factor (top_h)")

@@ -161,6 +161,24 @@ int monde_moe_ffn_fwd(const monde_problem* p, const void* x_perm,
 int monde_combine(const monde_problem* p, const void* y_perm, const int32_t* inv_perm,
                   const float* topk_w, void* out, void* stream);
 
+/* Expert FFN with the combine folded into its last store, for top-1 routing (one expert per
+ * token: the sum over experts has a single term, so no order of additions is lost).
+ * Paper: Section 2.1 (expert outputs are weighted by the gate and re-organised into the original
+ * token order); Section 3.4 (kernels fuse what follows a GEMM into it, as gemm+relu does).
+ *   for e with counts[e] > 0, rows r in [offsets[e], offsets[e+1]), t = perm[r]:
+ *     out[t,:] = topk_w[t] * round_dtype(h[r,:] * W2[e]^T + b2[e])      (rounded once more to dtype)
+ * i.e. bit for bit what monde_moe_ffn_fwd followed by monde_combine writes to `out`; y_perm is
+ * never materialised.  Returns MONDE_ERR_UNSUPPORTED unless top_k == 1 and dtype is bf16.
+ * in : as monde_moe_ffn_fwd (the class lists are not needed), perm [A] as written by
+ *      monde_permute, topk_w [T,1] fp32
+ * out: out [T,d_model] (dtype)
+ */
+int monde_moe_ffn_combine_fwd(const monde_problem* p, const void* x_perm,
+                              const void* W1, const void* b1, const void* W2, const void* b2,
+                              const int32_t* counts, const int32_t* offsets, const uint8_t* cls,
+                              const int32_t* perm, const float* topk_w, void* out,
+                              void* ws, size_t ws_bytes, void* stream);
+
 /* Synchronises `stream`, then returns and clears the sticky device-side status word
  * kept in `ws` (MONDE_OK, or MONDE_ERR_TIMEOUT if a bounded wait inside a kernel gave
  * up; the outputs of that call are then undefined).  `site` (nullable, host pointer)

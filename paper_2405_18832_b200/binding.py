@@ -66,6 +66,9 @@ def lib() -> ctypes.CDLL:
                                         vp, ctypes.c_size_t, vp]
         L.monde_moe_ffn_fwd_static_ws.restype = ctypes.c_int
         L.monde_moe_ffn_fwd_static_ws.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, i32p, i32p, i32p, vp, vp]
+        L.monde_moe_ffn_combine_fwd.restype = ctypes.c_int
+        L.monde_moe_ffn_combine_fwd.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, vp, i32p, f32p, vp, vp,
+                                                ctypes.c_size_t, vp]
         L.monde_combine.restype = ctypes.c_int
         L.monde_combine.argtypes = [pp, vp, i32p, f32p, vp, vp]
         L.monde_poll_device_status.restype = ctypes.c_int
@@ -139,6 +142,15 @@ def monde_moe_ffn_fwd(p, x_perm, W1, b1, W2, b2, counts, offsets, cls, hot_ids, 
         _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
 
 
+def monde_moe_ffn_combine_fwd(p, x_perm, W1, b1, W2, b2, counts, offsets, cls, perm, topk_w, out, ws,
+                              stream=None) -> None:
+    """Expert FFN with the gate-weighted combine folded into its last store (top-1, bf16 only)."""
+    cp = c_problem(p)
+    _check("monde_moe_ffn_combine_fwd", lib().monde_moe_ffn_combine_fwd(
+        ctypes.byref(cp), _ptr(x_perm), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(counts), _ptr(offsets),
+        _ptr(cls), _ptr(perm), _ptr(topk_w), _ptr(out), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
 STATIC_WS_BYTES = 32 << 20
 
 
@@ -194,11 +206,18 @@ class LayerBuffers:
         self.x_dev = torch.empty((T, d), dtype=dt, device=device)   # staging for host inputs
 
 
-def moe_ffn_layer_forward(p, x, Wg, bg, W1, b1, W2, b2, buf: LayerBuffers, stream=None) -> torch.Tensor:
-    """route -> permute -> expert FFN (hot + cold) -> combine, all enqueued on one stream."""
+def moe_ffn_layer_forward(p, x, Wg, bg, W1, b1, W2, b2, buf: LayerBuffers, stream=None,
+                          fuse_combine: bool = False) -> torch.Tensor:
+    """route -> permute -> expert FFN (hot + cold) -> combine, all enqueued on one stream.
+    `fuse_combine` (top-1 bf16 problems) takes the three-call form: the FFN's last store applies the
+    gate weight and writes `out` directly, same bytes, no y_perm."""
     monde_route(p, x, Wg, bg, buf.topk_idx, buf.topk_w, buf.counts, buf.offsets, buf.cls, buf.hot_ids,
                 buf.cold_ids, buf.n_hot_cold, buf.probs, buf.ws, stream)
     monde_permute(p, x, buf.topk_idx, buf.offsets, buf.perm, buf.inv_perm, buf.x_perm, buf.ws, stream)
+    if fuse_combine:
+        monde_moe_ffn_combine_fwd(p, buf.x_perm, W1, b1, W2, b2, buf.counts, buf.offsets, buf.cls, buf.perm,
+                                  buf.topk_w, buf.out, buf.ws, stream)
+        return buf.out
     monde_moe_ffn_fwd(p, buf.x_perm, W1, b1, W2, b2, buf.counts, buf.offsets, buf.cls, buf.hot_ids,
                       buf.cold_ids, buf.n_hot_cold, buf.y_perm, buf.ws, stream)
     monde_combine(p, buf.y_perm, buf.inv_perm, buf.topk_w, buf.out, stream)

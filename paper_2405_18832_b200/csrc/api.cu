@@ -152,6 +152,24 @@ int monde_moe_ffn_fwd(const monde_problem* p, const void* x_perm,
     return launch_ffn_bf16(*p, x_perm, W1, b1, W2, b2, counts, offsets, cls, y_perm, ws, s);
 }
 
+int monde_moe_ffn_combine_fwd(const monde_problem* p, const void* x_perm,
+                              const void* W1, const void* b1, const void* W2, const void* b2,
+                              const int32_t* counts, const int32_t* offsets, const uint8_t* cls,
+                              const int32_t* perm, const float* topk_w, void* out,
+                              void* ws, size_t ws_bytes, void* stream) {
+    int st = check_problem(p);
+    if (st != MONDE_OK) return st;
+    if (p->top_k != 1 || p->dtype != MONDE_BF16 || force_simt()) return MONDE_ERR_UNSUPPORTED;
+    if (p->T == 0) return MONDE_OK;
+    if (!x_perm || !W1 || !W2 || !counts || !offsets || !cls || !perm || !topk_w || !out) return MONDE_ERR_INVALID_ARG;
+    if (!aligned16(x_perm) || !aligned16(W1) || !aligned16(W2) || !aligned16(out) || !aligned16(b1) || !aligned16(b2))
+        return MONDE_ERR_INVALID_ARG;
+    if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
+    if ((st = check_arch()) != MONDE_OK) return st;
+    return launch_ffn_bf16(*p, x_perm, W1, b1, W2, b2, counts, offsets, cls, nullptr, ws,
+                           static_cast<cudaStream_t>(stream), perm, topk_w, out);
+}
+
 int monde_combine(const monde_problem* p, const void* y_perm, const int32_t* inv_perm,
                   const float* topk_w, void* out, void* stream) {
     int st = check_problem(p);

@@ -145,7 +145,8 @@ int launch_linear_simt(int dtype, int act_or_neg1, int E, int K, int N, const vo
 // weight-streaming kernel.
 int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, const void* b1,
                     const void* W2, const void* b2, const int32_t* counts, const int32_t* offsets,
-                    const uint8_t* cls, void* y_perm, void* ws, cudaStream_t s);
+                    const uint8_t* cls, void* y_perm, void* ws, cudaStream_t s,
+                    const int32_t* fuse_perm = nullptr, const float* fuse_w = nullptr, void* fuse_out = nullptr);
 
 // Process-wide count of kernels this library has launched (diagnostic).
 void count_launches(int n);

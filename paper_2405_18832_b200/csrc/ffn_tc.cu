@@ -98,6 +98,9 @@ struct FfnParams {
     int32_t* part_done;    // per cold second-layer tile: partial tiles finished
     float* partials;       // [tile][split][cold_tile tokens][128 features] fp32
     int32_t* ready;        // per token tile: first-layer units finished
+    const int32_t* fuse_perm;    // fused combine (top-1): assignment id of every row; null = store y
+    const float* fuse_w;         // gate weight per assignment
+    __nv_bfloat16* fuse_out;     // out [T, d_model]
     unsigned long long* trace;   // diagnostic timeline (null in normal use): [cta][unit slot][8]
     int trace_slots;
 };
@@ -874,12 +877,27 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             // One group = 16 tokens.  mode: 0 first layer (activation), 1 second layer, 2 second
             // layer finishing a K-split tile (adds the partial tiles), 3 partial tile (fp32 store).
             const int mode = un.layer == 0 ? 0 : (u_nsplit == 1 ? 1 : (is_partial ? 3 : 2));
+            const bool fused = P.fuse_out != nullptr && (mode == 1 || mode == 2);
             auto drain16 = [&](const uint32_t (&v)[16], int c0) {
                 if (mode == 3) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         part[(u_split * cold_tile + c0 + j) * kTileRows] = __uint_as_float(v[j]);
                     return;
+                }
+                // fused combine: the token and gate weight of the two rows this thread stores are
+                // fetched now and used after the transpose
+                int f_tok[2] = {0, 0};
+                float f_w[2] = {0.0f, 0.0f};
+                if (fused) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const int r = rd_row + half * 8;
+                        if (c0 + r < u_rows) {
+                            f_tok[half] = __ldg(P.fuse_perm + u_row0 + c0 + r);     // top-1: assignment id = token id
+                            f_w[half] = __ldg(P.fuse_w + f_tok[half]);
+                        }
+                    }
                 }
                 __nv_bfloat16* sb = stg_set + (grp & 1) * (16 * kTileRows) + q * 32 + lane;
                 if (mode == 0) {
@@ -914,7 +932,22 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     const int r = rd_row + half * 8;
                     if (col_ok && c0 + r < u_rows) {
                         const uint4 val = *reinterpret_cast<const uint4*>(rb + r * kTileRows + rd_col);
-                        *reinterpret_cast<uint4*>(out + static_cast<int64_t>(u_row0 + c0 + r) * N + n0 + rd_col) = val;
+                        if (fused) {
+                            // out[token] = gate weight x the bf16-rounded expert output, rounded once more:
+                            // the bytes monde_combine would produce from y_perm
+                            const uint32_t w4[4] = {val.x, val.y, val.z, val.w};
+                            uint32_t o4[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float lo = __uint_as_float(w4[i] << 16), hi = __uint_as_float(w4[i] & 0xFFFF0000u);
+                                const __nv_bfloat162 pr = __floats2bfloat162_rn(fmaf(f_w[half], lo, 0.0f), fmaf(f_w[half], hi, 0.0f));
+                                o4[i] = *reinterpret_cast<const uint32_t*>(&pr);
+                            }
+                            *reinterpret_cast<uint4*>(P.fuse_out + static_cast<int64_t>(f_tok[half]) * N + n0 + rd_col) =
+                                make_uint4(o4[0], o4[1], o4[2], o4[3]);
+                        } else {
+                            *reinterpret_cast<uint4*>(out + static_cast<int64_t>(u_row0 + c0 + r) * N + n0 + rd_col) = val;
+                        }
                     }
                 }
             };
@@ -1049,7 +1082,8 @@ int sm_count() {
 
 int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, const void* b1,
                     const void* W2, const void* b2, const int32_t* counts, const int32_t* offsets,
-                    const uint8_t* cls, void* y_perm, void* ws, cudaStream_t s) {
+                    const uint8_t* cls, void* y_perm, void* ws, cudaStream_t s, const int32_t* fuse_perm,
+                    const float* fuse_w, void* fuse_out) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
@@ -1106,6 +1140,9 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.part_done = reinterpret_cast<int32_t*>(base + L.part_done_off);
     P.partials = reinterpret_cast<float*>(base + L.partials_off);
     P.ready = reinterpret_cast<int32_t*>(base + WsLayout::kTiles);
+    P.fuse_perm = fuse_perm;
+    P.fuse_w = fuse_w;
+    P.fuse_out = static_cast<__nv_bfloat16*>(fuse_out);
     P.trace = g_trace;
     P.trace_slots = g_trace_slots;
     FfnMaps M;

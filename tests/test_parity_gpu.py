@@ -199,3 +199,31 @@ def test_host_pipeline_matches_step_by_step_results():
         torch.cuda.synchronize()
         assert torch.equal(o, ref.cpu())
     assert not torch.equal(outs[0], outs[1])
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "ragged_top1"])
+def test_fused_combine_gives_the_bytes_of_the_four_call_form(name):
+    # top-1: the FFN's last store applies the gate weight and writes `out`; must equal ffn + combine bit for bit
+    w = (_wl("ragged_top1", T=777, d_model=320, d_ff=832, E=9, hot_threshold=70, zipf_alpha=1.3, act="gelu")
+         if name == "ragged_top1" else S.config(name))
+    p = w.problem
+    g = S.generate(w)
+    dev = P.to_device(g)
+    weights = (dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"])
+    buf = B.LayerBuffers(p)
+    ref = B.moe_ffn_layer_forward(p, dev["x"], *weights, buf).clone()
+    buf.out.zero_()
+    buf.y_perm.fill_(float("nan"))          # the fused form must not depend on y_perm
+    got = B.moe_ffn_layer_forward(p, dev["x"], *weights, buf, fuse_combine=True)
+    B.monde_poll_device_status(buf.ws)
+    assert torch.equal(got, ref)
+
+
+def test_fused_combine_refuses_top2():
+    w = _wl("top2", T=64, top_k=2)
+    p = w.problem
+    dev = P.to_device(S.generate(w))
+    buf = B.LayerBuffers(p)
+    with pytest.raises(B.MondeError):
+        B.moe_ffn_layer_forward(p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"], buf,
+                                fuse_combine=True)
