@@ -15,14 +15,18 @@
 // A unit covers two 128-feature tiles that share one token tile (the token tile is the
 // operand that every feature tile re-reads through L2, so pairing halves that traffic).
 //   hot : token tile <= 256 (full-rate 128 x 256 MMAs).  For d_model >= 1536 a unit
-//         takes two feature tiles: 3 stages of 64 KB, and the two accumulators fill all 512
-//         TMEM columns, so the epilogue is not overlapped with the next unit's MMAs - cheaper
-//         than re-reading a 32 KB token tile per 16 KB weight tile.  For smaller layers the
-//         exposed epilogue and the halved unit count cost more than they save: one feature
-//         tile per unit, 4 stages of 48 KB, two accumulator buffers;
-//   cold: token tile = threshold-1 rounded up to 16 (at most 64), 4 or 5 stages of 34-40 KB,
-//         two accumulator buffers -> a deep queue of weight bytes in flight per SM; the tensor
-//         core idles most of the time and HBM sets the pace.
+//         takes two feature tiles (three 32 KB weight stages, three 32 KB token stages), and
+//         the two accumulators fill all 512 TMEM columns, so the epilogue is not overlapped
+//         with the next unit's MMAs - cheaper than re-reading a 32 KB token tile per 16 KB
+//         weight tile.  For smaller layers the exposed epilogue and the halved unit count
+//         cost more than they save: one feature tile per unit (six 16 KB weight stages, three
+//         32 KB token stages), two accumulator buffers;
+//   cold: token tile = threshold-1 rounded up to 16 (at most 64), two feature tiles per unit,
+//         five 32 KB weight stages and four small token stages, two accumulator buffers -> a
+//         deep queue of weight bytes in flight per SM; the tensor core idles most of the time
+//         and HBM sets the pace.
+// Weight tiles (from HBM, long latency) and token tiles (from L2, re-read by every feature
+// tile) have separate rings and separate producer warps.
 // Work units (expert, 128-feature tile, token tile) form one ordered list: hot first
 // layer, hot second layer, cold first layer, cold second layer.  One persistent CTA per SM
 // takes the next unit from a device-wide counter.  A second-layer unit needs the hidden
@@ -39,6 +43,9 @@
 // loads, warp 1 issues MMAs and owns the TMEM allocation, warps 2-5 and 8-11 drain the
 // accumulator (bias + activation fused) while the next unit's MMAs run into the second
 // accumulator buffer, warp 6 publishes finished rows.  Counts never travel to the host.
+// Variants of the same kernel: CTA pairs (template parameter kPair: clusters of two CTAs issue
+// one 256-row MMA, tcgen05 cta_group::2; opt-in), and a last store that applies the gate weight
+// and writes the layer output in token order (top-1 routing, monde_moe_ffn_combine_fwd).
 #include <cuda.h>
 
 #include <algorithm>
