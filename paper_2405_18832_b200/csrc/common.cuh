@@ -22,18 +22,23 @@ struct WsLayout {
     static constexpr size_t kCountersBytes = 15 * 1024;
     static constexpr size_t kTiles = 16 * 1024; // work lists built on the device
     static constexpr size_t kTilesBytes = 112 * 1024;
-    static constexpr size_t kHidden = 128 * 1024;  // h [A, d_ff] in the problem dtype
+    static constexpr size_t kPartDone = 128 * 1024;   // int32 per cold second-layer tile: partial tiles finished
+    static constexpr size_t kPartDoneBytes = 128 * 1024;
+    static constexpr size_t kHidden = 256 * 1024;  // h [A, d_ff] in the problem dtype
     size_t hidden_bytes;
     int n_split;            // K-splits of a cold second-layer unit
-    size_t part_done_off;   // int32 per cold second-layer tile (zero between calls)
+    size_t part_done_off;   // = kPartDone: inside the header, so it is zero whatever problem used the buffer before
     size_t part_done_bytes;
     size_t partials_off;    // fp32 partial tiles of the K-split cold second-layer units
     size_t partials_bytes;
     size_t total;
 };
 // The header (first kHidden bytes) holds everything that must be zero between calls: the
-// status word, the CTA ticket (kCounters) and one int32 per token tile that counts finished
-// first-layer units (kTiles).  A <= kMaxAssignments keeps the token-tile counters inside it.
+// status word, the CTA ticket (kCounters), one int32 per token tile that counts finished
+// first-layer units (kTiles) and one per cold second-layer tile that counts finished partial
+// tiles (kPartDone).  Its layout does not depend on the problem, so problems of different shapes
+// may take turns on one workspace.  A <= kMaxAssignments keeps the token-tile counters inside
+// it; problems with more cold second-layer tiles than kPartDone holds run without the K-split.
 constexpr int64_t kMaxAssignments = 1 << 20;
 static_assert(4 * (kMaxAssignments / 64 + 2 * 256 + 64) <= 112 * 1024, "token-tile counters overflow the header");
 
@@ -59,11 +64,11 @@ inline WsLayout ws_layout(const monde_problem& p) {
     const int kb2 = p.d_ff / 64;                              // every sub-unit must own at least one K block
     while (split > 1 && (split - 1) * ((kb2 + split - 1) / split) >= kb2) --split;
     size_t part = cold_tiles * (split - 1) * ct * 128 * 4;
-    if (part > (size_t(1) << 30)) { split = 1; part = 0; }
+    if (part > (size_t(1) << 30) || cold_tiles * 4 > WsLayout::kPartDoneBytes) { split = 1; part = 0; }
     l.n_split = split;
-    l.part_done_off = WsLayout::kHidden + l.hidden_bytes;
+    l.part_done_off = WsLayout::kPartDone;
     l.part_done_bytes = split > 1 ? (cold_tiles * 4 + 1023) / 1024 * 1024 : 0;
-    l.partials_off = l.part_done_off + l.part_done_bytes;
+    l.partials_off = WsLayout::kHidden + l.hidden_bytes;
     l.partials_bytes = part;
     l.total = l.partials_off + l.partials_bytes + 1024;
     return l;

@@ -55,14 +55,11 @@ extern "C" int monde_moe_ffn_fwd_static_ws(const monde_problem* p, const void* x
     void* ws = nullptr;
     if ((st = static_ws_ptr(&ws)) != MONDE_OK) return st;
     // The array keeps whatever the previous call left.  Everything the kernels expect to find
-    // at zero lives in the header and in the per-tile split-K counters: clear both, in stream
-    // order, before the launch.  The hidden activations and partial tiles are fully rewritten
-    // before they are read.
+    // at zero lives in the header (status, tickets, dependency counters, split-K counters):
+    // clear it, in stream order, before the launch.  The hidden activations and partial tiles
+    // are fully rewritten before they are read.
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, monde::WsLayout::kHidden, s) != cudaSuccess) return MONDE_ERR_CUDA;
-    if (L.part_done_bytes != 0 &&
-        cudaMemsetAsync(static_cast<char*>(ws) + L.part_done_off, 0, L.part_done_bytes, s) != cudaSuccess)
-        return MONDE_ERR_CUDA;
     return monde_moe_ffn_fwd(p, x_perm, W1, b1, W2, b2, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold, y_perm,
                              ws, kStaticWsBytes, stream);
 }

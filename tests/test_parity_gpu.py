@@ -227,3 +227,24 @@ def test_fused_combine_refuses_top2():
     with pytest.raises(B.MondeError):
         B.moe_ffn_layer_forward(p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"], buf,
                                 fuse_combine=True)
+
+
+def test_one_workspace_serves_alternating_problems():
+    # every call leaves the workspace header at zero, so problems of different shapes (different token-tile
+    # counts, K-splits, classes) may take turns on one buffer sized for the largest
+    wa = _wl("alt_a", T=500, d_model=256, d_ff=1024, E=12, top_k=2, renormalize=1, hot_threshold=40, zipf_alpha=1.2)
+    wb = _wl("alt_b", T=90, d_model=384, d_ff=768, E=32, top_k=1, hot_threshold=16, act="gelu")
+    runs = []
+    for w in (wa, wb):
+        g = S.generate(w)
+        dev = P.to_device(g)
+        fresh = P.run_gpu(w.problem, dev, want_probs=False).out.clone()
+        runs.append((w.problem, dev, fresh))
+    shared = torch.zeros(max(B.monde_workspace_bytes(p) for p, _, _ in runs), dtype=torch.uint8, device="cuda")
+    for p, dev, fresh in runs + runs[::-1] + runs:
+        buf = B.LayerBuffers(p)
+        buf.ws = shared
+        out = B.moe_ffn_layer_forward(p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"], buf)
+        B.monde_poll_device_status(shared)
+        assert torch.equal(out, fresh)
+    assert int(shared[:128 * 1024].to(torch.int32).sum()) == 0      # header back at zero
