@@ -368,6 +368,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     }
     pdl_wait();
 
+    // Every unit, the first included, comes from the device-wide counter: a unit is only ever held
+    // by a CTA that is running, so a launch whose CTAs are not all resident at once (another
+    // kernel holding some SMs) still cannot wait on a unit that nobody is working on.  The draw is
+    // issued here and its answer used after the unit table is built, which hides the round trip.
+    int first_draw = 0;
+    if (warp == 0 && lane == 0 && (!kPair || cluster_ctarank() == 0)) first_draw = atomicAdd(P.next_unit, 1);
+
     // ---- unit table from the router's outputs -----------------------------------------------
     // Thread e reads expert e's class, count and offset (independent loads: one round trip to
     // memory instead of the three that following n_hot_cold -> id lists -> counts would take) and
@@ -449,8 +456,6 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     // accumulator-free barriers that the MMA issuer waits on live in the leader only).
     const uint32_t rank = kPair ? cluster_ctarank() : 0u;
     const uint32_t bar0_leader = kPair ? map_to_cta(bar0, 0) : bar0;
-    const int n_workers = kPair ? static_cast<int>(gridDim.x) / 2 : static_cast<int>(gridDim.x);
-    const int worker = kPair ? static_cast<int>(blockIdx.x) / 2 : static_cast<int>(blockIdx.x);
     const int tt_all = ut.tt_prefix[ut.n_all];
     const int tt_hot = ut.tt_prefix[ut.n_hot];
     ut.kblocks1 = P.d_model / kBlockK;
@@ -542,24 +547,31 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 mbar_arrive(q_full(slot));          // release: the record is visible to whoever acquires
                 return true;
             };
-            // The first unit of worker w (a CTA, or a CTA pair) is unit w: no round trip to the counter
-            // before the first load.  The counter hands out the rest.  In a CTA pair the
+            // In a CTA pair the
             // leader draws from the counter and posts the index into the other CTA's mailbox (a
             // remote store released by a remote mbarrier arrival).  The other CTA's loads gate the
             // leader's MMAs, so it is never more than five draws behind and eight slots suffice.
             int draws = 0;
-            auto draw = [&]() -> int { return atomicAdd(P.next_unit, 1) + n_workers; };
+            auto draw = [&]() -> int {
+                if (draws == 0) return first_draw;      // drawn before the unit table was built
+                return atomicAdd(P.next_unit, 1);
+            };
             auto take_next = [&]() -> int {
-                if (!kPair) return draw();
+                if (!kPair) {
+                    const int idx = draw();
+                    ++draws;
+                    return idx;
+                }
                 const int slot = draws % kMailSlots;
                 const uint32_t parity = (draws / kMailSlots) & 1;
-                ++draws;
                 if (rank == 0) {
                     const int idx = draw();
+                    ++draws;
                     st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(mail) + slot), 1), static_cast<uint32_t>(idx));
                     mbar_arrive_cluster(map_to_cta(mail_bar(slot), 1));
                     return idx;
                 }
+                ++draws;
                 if (!mbar_wait_cluster(mail_bar(slot), parity, abort_flag, kWaitLimitNs)) {
                     report_timeout(P.status, abort_flag, kSiteQueue);
                     return 0x7fffffff;
@@ -567,7 +579,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 return mail[slot];
             };
             Unit cur, nxt;
-            const int u = worker;
+            const int u = take_next();
             cur.id = -1;
             if (u < ut.total_units) cur = ut.decode(u);
             ok = push_unit(0, cur);

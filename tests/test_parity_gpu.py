@@ -248,3 +248,22 @@ def test_one_workspace_serves_alternating_problems():
         B.monde_poll_device_status(shared)
         assert torch.equal(out, fresh)
     assert int(shared[:128 * 1024].to(torch.int32).sum()) == 0      # header back at zero
+
+
+def test_two_layers_on_two_streams_at_once():
+    # two persistent launches that cannot both be fully resident: each must still finish (a unit is only
+    # ever held by a running CTA) and give the results of running alone
+    wa = _wl("conc_a", T=2000, d_model=512, d_ff=2048, E=16, top_k=2, renormalize=1, hot_threshold=64, zipf_alpha=1.2)
+    wb = _wl("conc_b", T=1500, d_model=768, d_ff=1536, E=24, top_k=1, hot_threshold=48, zipf_alpha=1.0, act="gelu")
+    jobs = []
+    for w in (wa, wb):
+        dev = P.to_device(S.generate(w))
+        alone = P.run_gpu(w.problem, dev, want_probs=False).out.clone()
+        jobs.append((w.problem, dev, alone, B.LayerBuffers(w.problem), torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    for _ in range(10):
+        for p, dev, _, buf, st in jobs:
+            B.moe_ffn_layer_forward(p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"], buf, st)
+    for p, dev, alone, buf, st in jobs:
+        B.monde_poll_device_status(buf.ws, st)
+        assert torch.equal(buf.out, alone)
