@@ -267,3 +267,33 @@ def test_two_layers_on_two_streams_at_once():
     for p, dev, alone, buf, st in jobs:
         B.monde_poll_device_status(buf.ws, st)
         assert torch.equal(buf.out, alone)
+
+
+def test_layer_captured_in_a_cuda_graph_replays_with_new_tokens():
+    # decode loops capture the four calls once and replay them: the launches (programmatic dependent launch
+    # included) must be capturable and every replay must leave the workspace ready for the next
+    w = _wl("graph", T=48, d_model=256, d_ff=1024, E=16, top_k=2, renormalize=1, hot_threshold=12, zipf_alpha=1.0)
+    p = w.problem
+    g = S.generate(w)
+    dev = P.to_device(g)
+    weights = (dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"])
+    buf = B.LayerBuffers(p)
+    x_static = dev["x"].clone()
+    B.moe_ffn_layer_forward(p, x_static, *weights, buf)          # first call outside capture (one-time set-up)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            B.moe_ffn_layer_forward(p, x_static, *weights, buf, side)
+    eager = B.LayerBuffers(p)
+    gen = torch.Generator().manual_seed(9)
+    for i in range(4):
+        x_new = (g["x"].float() * (1.0 + 0.5 * i) + 0.02 * torch.randn(g["x"].shape, generator=gen)).to(g["x"].dtype).cuda()
+        x_static.copy_(x_new)
+        graph.replay()
+        torch.cuda.synchronize()
+        ref = B.moe_ffn_layer_forward(p, x_new, *weights, eager)
+        B.monde_poll_device_status(eager.ws)
+        assert torch.equal(buf.out, ref)
+    B.monde_poll_device_status(buf.ws)
