@@ -297,3 +297,14 @@ def test_layer_captured_in_a_cuda_graph_replays_with_new_tokens():
         B.monde_poll_device_status(eager.ws)
         assert torch.equal(buf.out, ref)
     B.monde_poll_device_status(buf.ws)
+
+
+def test_maximum_assignment_count():
+    # T * top_k = 2^20, the stated limit: routing, permutation and row gather bit-exact in full (two-level
+    # recount over 512 super-chunks), expert outputs on a sample; 16384 assignments per expert on average
+    w = _wl("max_A", T=1 << 19, d_model=64, d_ff=128, E=64, top_k=2, renormalize=1, hot_threshold=64,
+            zipf_alpha=0.8, bias="none")
+    g = S.generate(w)
+    dev = P.to_device(g)
+    r = P.check_sampled(w, g, dev, n_tokens=256)
+    assert int(r.route.counts.sum()) == 1 << 20 and r.route.n_hot_cold[0] == 64
