@@ -308,3 +308,18 @@ def test_maximum_assignment_count():
     dev = P.to_device(g)
     r = P.check_sampled(w, g, dev, n_tokens=256)
     assert int(r.route.counts.sum()) == 1 << 20 and r.route.n_hot_cold[0] == 64
+
+
+def test_wide_hot_units_with_odd_and_half_feature_tiles():
+    # d_model >= 1536 selects two-feature-tile hot units; 1664 = 13 tiles and 1728 = 13.5 tiles leave a last
+    # unit with one tile and a tile with 64 valid features, in both layers and both classes
+    w = _wl("wide_odd", T=640, d_model=1664, d_ff=1728, E=6, top_k=2, renormalize=1, hot_threshold=100,
+            zipf_alpha=1.4, act="gelu")
+    r = P.check_full(w)
+    assert r.route.n_hot_cold[0] >= 2 and r.route.n_hot_cold[1] >= 1
+
+
+def test_wide_hot_units_with_odd_and_half_feature_tiles_on_cta_pairs(cta_pairs):
+    w = _wl("wide_odd_pairs", T=640, d_model=1664, d_ff=1728, E=6, top_k=2, renormalize=1, hot_threshold=100,
+            zipf_alpha=1.4, act="gelu")
+    P.check_full(w)
