@@ -70,7 +70,9 @@ typedef struct {
  * layer; calls that share a buffer must be ordered on one stream.  The caller
  * zero-fills it ONCE after allocating it (it holds the sticky status word and
  * counters that every call leaves at zero again); its contents need not be
- * preserved otherwise.  Returns 0 for an invalid problem. */
+ * preserved otherwise.  Problems of different shapes may take turns on one buffer that
+ * is large enough for each of them; calls that run at the same time (different streams)
+ * need a buffer each.  Returns 0 for an invalid problem. */
 size_t monde_workspace_bytes(const monde_problem* p);
 
 const char* monde_status_string(int status);
