@@ -43,7 +43,7 @@ UNIT = "tokens/s"
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures
 # summarised in profiles/expert_ffn_kernel_C1_C2.md (None where no capture exists).
-NCU_TRAFFIC_BYTES = {"C1": 628.2e6, "C2": 459.3e6, "C3": None}
+NCU_TRAFFIC_BYTES = {"C1": 630.3e6, "C2": 459.8e6, "C3": None}
 
 
 def measured_peaks():
