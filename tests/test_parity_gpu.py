@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import parity as P
 from paper_2405_18832_b200 import binding as B
 from paper_2405_18832_b200 import synthetic as S
@@ -323,3 +324,52 @@ def test_wide_hot_units_with_odd_and_half_feature_tiles_on_cta_pairs(cta_pairs):
     w = _wl("wide_odd_pairs", T=640, d_model=1664, d_ff=1728, E=6, top_k=2, renormalize=1, hot_threshold=100,
             zipf_alpha=1.4, act="gelu")
     P.check_full(w)
+
+
+def _random_workloads(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        big = rng.random() < 0.2
+        d_model = int(64 * (rng.integers(24, 37) if big else rng.integers(1, 13)))
+        d_ff = int(64 * rng.integers(1, 17 if not big else 9))
+        E = int(rng.integers(1, 41))
+        top_k = int(rng.integers(1, min(E, 4) + 1))
+        out.append(_wl(f"fuzz{i}", T=int(rng.integers(1, 300 if big else 1500)), d_model=d_model, d_ff=d_ff, E=E,
+                       top_k=top_k, renormalize=int(rng.integers(0, 2)), hot_threshold=int(rng.choice([1, 4, 16, 64, 300])),
+                       zipf_alpha=float(rng.choice([0.0, 0.7, 1.2, 1.6])), act=str(rng.choice(["relu", "gelu"])),
+                       bias=str(rng.choice(["random", "none"])), seed=100 + i))
+    return out
+
+
+def test_random_shapes_on_one_shared_workspace():
+    # 24 seeded random problems (sizes, expert counts, k, thresholds, skew, activation, biases), one after the
+    # other on a single workspace, the expert FFN alternately on single CTAs and on CTA pairs, top-1 problems
+    # also through the fused-combine entry point; every one against the oracle element by element
+    ws = _random_workloads(24, seed=2024)
+    shared = torch.zeros(max(B.monde_workspace_bytes(w.problem) for w in ws), dtype=torch.uint8, device="cuda")
+    try:
+        for i, w in enumerate(ws):
+            p = w.problem
+            B.lib().monde_internal_set_ffn_pair(i % 2)
+            g = S.generate(w)
+            dev = P.to_device(g)
+            buf = B.LayerBuffers(p, want_probs=True)
+            buf.ws = shared
+            B.moe_ffn_layer_forward(p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"], buf)
+            B.monde_poll_device_status(shared)
+            r, pm = P.check_routing(p, g, buf)
+            y_ref = oracle.expert_ffn(pm.x_perm, oracle.experts_of_rows(r.offsets), S.as_numpy(g["W1"]), S.as_numpy(g["b1"]),
+                                      S.as_numpy(g["W2"]), S.as_numpy(g["b2"]), p.act)
+            P.check_close(f"{w.name} y_perm", P.widen(buf.y_perm), y_ref, p.dtype)
+            out_ref = oracle.combine(y_ref, pm.inv_perm, r.topk_w)
+            P.check_close(f"{w.name} out", P.widen(buf.out), out_ref, p.dtype)
+            if p.top_k == 1:
+                four_calls = buf.out.clone()
+                buf.out.zero_()
+                B.moe_ffn_layer_forward(p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"], buf,
+                                        fuse_combine=True)
+                B.monde_poll_device_status(shared)
+                assert torch.equal(buf.out, four_calls), w.name
+    finally:
+        B.lib().monde_internal_set_ffn_pair(-1)
