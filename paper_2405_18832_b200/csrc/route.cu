@@ -248,8 +248,11 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int kTilesPerWarp>   // 8-expert column tiles per warp: padded E = 32 * kTilesPerWarp
-__global__ void __launch_bounds__(512) route_mma_kernel(
+// kTilesPerWarp: 8-expert column tiles per warp, padded E = 32 * kTilesPerWarp.  kDeep: grids of at most
+// one CTA per SM keep the loads of several K steps in flight (about 128 registers); larger grids keep
+// two CTAs per SM (64 registers) and load a step at a time.
+template <int kTilesPerWarp, bool kDeep>
+__global__ void __launch_bounds__(512, (kDeep || kTilesPerWarp >= 8) ? 1 : 2) route_mma_kernel(
         int T_tokens, int d, int E, int k, int renorm, const __nv_bfloat16* __restrict__ x,
         const __nv_bfloat16* __restrict__ Wg, const float* __restrict__ bg, int32_t* __restrict__ topk_idx,
         float* __restrict__ topk_w, float* __restrict__ probs, const HistArgs hist) {
@@ -279,14 +282,30 @@ __global__ void __launch_bounds__(512) route_mma_kernel(
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[j][i] = 0.0f;
     const int steps = d / 32;               // 32 k per step: 4 lanes x 8 elements
-#pragma unroll 4
-    for (int s = kq; s < steps; s += 4) {
-        const uint4 a = xa[s * 4], b = xb[s * 4];
+    // Loads of several steps are issued together and the MMAs follow: a step at a time would put one
+    // trip to memory per step on the critical path of a kernel that is all latency.
+    constexpr int kBatch = (!kDeep || kTilesPerWarp >= 8) ? 1 : 20 / (2 + kTilesPerWarp);   // about 80 registers of loads in flight
+    for (int s0 = kq; s0 < steps; s0 += 4 * kBatch) {
+        uint4 a[kBatch], b[kBatch], w[kBatch][kTilesPerWarp];
 #pragma unroll
-        for (int j = 0; j < kTilesPerWarp; ++j) {
-            const uint4 w = wp[j][s * 4];
-            mma_bf16_16816(acc[j], a.x, b.x, a.y, b.y, w.x, w.y);
-            mma_bf16_16816(acc[j], a.z, b.z, a.w, b.w, w.z, w.w);
+        for (int i = 0; i < kBatch; ++i) {
+            const int s = s0 + 4 * i;
+            if (s < steps) {
+                a[i] = xa[s * 4];
+                b[i] = xb[s * 4];
+#pragma unroll
+                for (int j = 0; j < kTilesPerWarp; ++j) w[i][j] = wp[j][s * 4];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            if (s0 + 4 * i < steps) {
+#pragma unroll
+                for (int j = 0; j < kTilesPerWarp; ++j) {
+                    mma_bf16_16816(acc[j], a[i].x, b[i].x, a[i].y, b[i].y, w[i][j].x, w[i][j].y);
+                    mma_bf16_16816(acc[j], a[i].z, b[i].z, a[i].w, b[i].w, w[i][j].z, w[i][j].w);
+                }
+            }
         }
     }
     float* part = s_part + kq * (16 * kRow);
@@ -322,13 +341,29 @@ int launch_route_mma(const monde_problem& p, const void* x, const void* Wg, cons
                      float* topk_w, float* probs, const HistArgs& hist, cudaStream_t s) {
     constexpr int kSmem = 4 * 16 * (32 * kTilesPerWarp + 1) * 4;
     if (kSmem > 48 * 1024) {
-        static const cudaError_t attr = cudaFuncSetAttribute(route_mma_kernel<kTilesPerWarp>,
-                                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        static const cudaError_t attr = [] {
+            cudaError_t e = cudaFuncSetAttribute(route_mma_kernel<kTilesPerWarp, false>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+            return e != cudaSuccess ? e : cudaFuncSetAttribute(route_mma_kernel<kTilesPerWarp, true>,
+                                                               cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        }();
         if (attr != cudaSuccess) return MONDE_ERR_CUDA;
     }
-    launch_pdl(route_mma_kernel<kTilesPerWarp>, dim3((p.T + 15) / 16), dim3(512), kSmem, s,
-        p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),
-        static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs, hist);
+    const int grid = (p.T + 15) / 16;
+    static const int sms = [] {
+        int dev = 0, v = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+        return v > 0 ? v : 148;
+    }();
+    if (grid <= sms)
+        launch_pdl(route_mma_kernel<kTilesPerWarp, true>, dim3(grid), dim3(512), kSmem, s,
+            p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),
+            static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs, hist);
+    else
+        launch_pdl(route_mma_kernel<kTilesPerWarp, false>, dim3(grid), dim3(512), kSmem, s,
+            p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),
+            static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs, hist);
     return MONDE_OK;
 }
 
