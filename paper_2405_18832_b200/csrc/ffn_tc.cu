@@ -72,6 +72,7 @@ constexpr int kABytes = kTileRows * 128;
 constexpr int kMaxStagesA = 10;       // weight-tile ring
 constexpr int kMaxStagesB = 4;        // token-tile ring
 constexpr int kQueue = 4;            // unit ids in flight between the producer and the other roles
+constexpr int kClaimAhead = 6;       // K blocks still to load when the producer takes its next unit
 constexpr int kHotTokTile = 256;
 constexpr int kTilesPerUnit = 2;      // a unit covers two 128-feature tiles that share one token tile
 constexpr int kTileBytes = 192 * 1024;
@@ -611,8 +612,10 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 const bool trace_on = P.trace != nullptr;
                 bool next_ready = false;
                 for (int kb = kb0; kb < kb1; kb += kKps) {
-                    if (!next_ready && (kb - kb0 == 2 || kb + kKps >= kb1)) {
-                        // take, decode and publish the next unit while this one's loads are in flight
+                    if (!next_ready && (kb1 - kb <= kClaimAhead || kb + kKps >= kb1)) {
+                        // take, decode and publish the next unit while this one's last loads are in flight
+                        // (not earlier: a unit claimed at the start of a long one would sit unworked for
+                        // the whole of it while other SMs run out of units of its kind)
                         nxt.id = -1;
                         if (u_ahead < ut.total_units) {
                             nxt = ut.decode(u_ahead);
