@@ -1084,9 +1084,8 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, ui
     const cuuint64_t strides[1] = {cols * 2};
     const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    static const int promo = [] { const char* e = getenv("MONDE_L2PROMO"); return e ? atoi(e) : 3; }();
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, static_cast<CUtensorMapL2promotion>(promo),
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
