@@ -389,8 +389,11 @@ def run_ours(args, w):
         host = host_inputs(g)
         n_tok = pick_sample_tokens(w, host, 12.0)
         sec = oracle_sample_run(w, host, n_tok)
+        n_one = max(1, min(n_tok, int(n_tok / sec * 3.0 / max(oracle.usable_cores(), 1))))   # about 3 s on one thread
+        sec_one = oracle_sample_run(w, host, n_one, nthreads=1)
         cpu = {"value": n_tok / sec, "unit": UNIT, "cores": oracle.usable_cores(), "kind": "oracle",
-               "sample": f"whole layer on the first {n_tok} of {p.T} tokens, {sec:.1f} s"}
+               "sample": f"whole layer on the first {n_tok} of {p.T} tokens, {sec:.1f} s",
+               "one_thread": {"value": n_one / sec_one, "sample": f"first {n_one} tokens, {sec_one:.1f} s"}}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
