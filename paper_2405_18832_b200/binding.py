@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmonde.so")
 
 SYMBOLS = ("monde_workspace_bytes", "monde_status_string", "monde_route", "monde_classify_top_h", "monde_permute",
-           "monde_moe_ffn_fwd", "monde_moe_ffn_fwd_static_ws", "monde_combine", "monde_poll_device_status",
+           "monde_moe_ffn_fwd", "monde_moe_ffn_combine_fwd", "monde_moe_ffn_fwd_static_ws", "monde_combine", "monde_poll_device_status",
            "monde_kernel_launches")
 
 _DTYPE = {"f32": 0, "bf16": 1}
