@@ -332,7 +332,7 @@ def run_ours(args, w):
     e2e_serial_value = aggregate_tokens_per_s(p.T, world, serial_ms / args.steps)
     assert torch.equal(out_host, buf.out.cpu())
 
-    pipe = B.HostPipeline(p, depth=2)
+    pipe = B.HostPipeline(p, depth=2, device=dev)
     weights = (d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"])
     out_host.zero_()
     for _ in range(max(3, args.warmup)):
