@@ -64,6 +64,23 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
     for (int e = tid; e < kMaxExperts; e += kThreads) before[e] = 0;
     __syncthreads();
     pdl_wait();
+    // The rows this warp will copy are known before their positions are: their first vectors are
+    // requested now, so that trip to memory overlaps the recount and the rank computation.
+    constexpr int V = Vec16<T>::N;
+    constexpr int kIter = 3;                         // vectors per lane and row in flight
+    const int vec_per_row = d / V;
+    const uint4* src[kRowsPerWarp];
+    uint4 v[kIter][kRowsPerWarp];
+#pragma unroll
+    for (int r = 0; r < kRowsPerWarp; ++r) {
+        const int a = first + warp * kRowsPerWarp + r;
+        src[r] = a < A ? reinterpret_cast<const uint4*>(x + static_cast<int64_t>(a / k) * d) : nullptr;
+    }
+#pragma unroll
+    for (int it = 0; it < kIter; ++it)
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r)
+            if (src[r] != nullptr && lane + 32 * it < vec_per_row) v[it][r] = src[r][lane + 32 * it];
     const int recount_from = super_before != nullptr ? (first / kSuper) * kSuper : 0;
     if (super_before != nullptr)
         for (int e = tid; e < E; e += kThreads) before[e] = super_before[static_cast<size_t>(first / kSuper) * E + e];
@@ -107,26 +124,27 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
         if (lane < kChunk) row_pos[lane] = pos;
     }
     __syncthreads();
-    // Row gather with 16-byte accesses; the warp's rows advance together.
-    constexpr int V = Vec16<T>::N;
-    const int vec_per_row = d / V;
-    const uint4* src[kRowsPerWarp];
+    // Row gather with 16-byte accesses; the warp's rows advance together, kIter vectors per lane and
+    // row requested before any is stored (one trip to memory per batch, not per vector).
     uint4* dst[kRowsPerWarp];
 #pragma unroll
     for (int r = 0; r < kRowsPerWarp; ++r) {
-        const int idx = warp * kRowsPerWarp + r;
-        const int p = row_pos[idx];
-        src[r] = p >= 0 ? reinterpret_cast<const uint4*>(x + static_cast<int64_t>((first + idx) / k) * d) : nullptr;
+        const int p = row_pos[warp * kRowsPerWarp + r];
         dst[r] = p >= 0 ? reinterpret_cast<uint4*>(x_perm + static_cast<int64_t>(p) * d) : nullptr;
     }
-    for (int i = lane; i < vec_per_row; i += 32) {
-        uint4 v[kRowsPerWarp];
+    for (int i0 = lane; i0 < vec_per_row; i0 += 32 * kIter) {
+        if (i0 != lane) {      // the first batch is already in registers
 #pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r)
-            if (src[r] != nullptr) v[r] = src[r][i];
+            for (int it = 0; it < kIter; ++it)
 #pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r)
-            if (dst[r] != nullptr) dst[r][i] = v[r];
+                for (int r = 0; r < kRowsPerWarp; ++r)
+                    if (dst[r] != nullptr && i0 + 32 * it < vec_per_row) v[it][r] = src[r][i0 + 32 * it];
+        }
+#pragma unroll
+        for (int it = 0; it < kIter; ++it)
+#pragma unroll
+            for (int r = 0; r < kRowsPerWarp; ++r)
+                if (dst[r] != nullptr && i0 + 32 * it < vec_per_row) dst[r][i0 + 32 * it] = v[it][r];
     }
 }
 
