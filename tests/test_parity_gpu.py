@@ -373,3 +373,25 @@ def test_random_shapes_on_one_shared_workspace():
                 assert torch.equal(buf.out, four_calls), w.name
     finally:
         B.lib().monde_internal_set_ffn_pair(-1)
+
+
+def test_device_status_word_is_reported_and_cleared():
+    # the host side of the bounded-wait protocol, with the status word written from the host (no kernel is
+    # made to give up): the poll reports it with its site code, clears the whole header, and the workspace
+    # serves the next call
+    w = S.config("C0")
+    p = w.problem
+    dev = P.to_device(S.generate(w))
+    buf = P.run_gpu(p, dev, want_probs=False)
+    good = buf.out.clone()
+    hdr = buf.ws[:64].view(torch.int32)
+    hdr[0] = 6            # MONDE_ERR_TIMEOUT
+    hdr[1] = 5            # a site code
+    buf.ws[4096:4100] = 7  # stray counter contents that a half-finished call could leave in the header
+    with pytest.raises(B.MondeError) as err:
+        B.monde_poll_device_status(buf.ws)
+    assert "site 5" in str(err.value) and err.value.status == 6
+    assert int(buf.ws[:256 * 1024].to(torch.int32).sum()) == 0
+    out = B.moe_ffn_layer_forward(p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"], buf)
+    B.monde_poll_device_status(buf.ws)
+    assert torch.equal(out, good)
