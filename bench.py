@@ -2,10 +2,13 @@
 """Benchmark of the MoE FFN layer forward (route -> permute -> hot/cold expert FFN ->
 combine) on synthetic Switch / NLLB-shaped workloads.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1|C2|C3] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C3|C2|C1|HOTPROBE|C4:...] [--impl ours|reference]
 
 One JSON line on stdout (rank 0).  A step is one pass of the whole layer over one
-batch of T tokens.  `value` is tokens/s with inputs resident in HBM; `e2e` is the
+batch of T tokens.  The headline workload is C3, the NLLB-MoE-like layer (the largest
+stated single-GPU configuration); the same line carries, under `per_workload`, the same
+measurements for C2 (the decode step the cold-streaming target is quoted on), C1 and the
+compute-bound probe of the hot tiling (`--no-sub-workloads` leaves them out).  `value` is tokens/s with inputs resident in HBM; `e2e` is the
 same layer called with the step's tokens in pinned host memory (H2D copy of x and
 D2H copy of the output for every step inside the timed region; `binding.HostPipeline`
 overlaps the copies of neighbouring steps with the compute, `e2e.serial_value` is the
@@ -41,9 +44,17 @@ from paper_2405_18832_b200 import synthetic as S  # noqa: E402
 METRIC = "moe_ffn_layer_tokens_per_s"
 UNIT = "tokens/s"
 
-# DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures
-# summarised in profiles/expert_ffn_kernel_C1_C2.md (None where no capture exists).
-NCU_TRAFFIC_BYTES = {"C1": 630.3e6, "C2": 459.8e6, "C3": None}
+# DRAM bytes (read + write) of one launch of the dominant kernel.  Not measured in this run: taken
+# from the ncu captures summarised under profiles/ (a profiler cannot run inside a timed benchmark).
+# C3's weights (8.6 GB) are above the size a capture may hold, so its figure is C2's measured
+# traffic per activated expert's weight byte (459.8 MB for 27 experts x 16.78 MB = 1.0150) times
+# C3's own weight bytes; traffic grows in proportion because DRAM reads are the weights read once.
+NCU_TRAFFIC = {
+    "C1": (630.3e6, "profiles/expert_ffn_kernel_C1_C2.md (ncu, one launch), not this run"),
+    "C2": (459.8e6, "profiles/expert_ffn_kernel_C1_C2.md (ncu, one launch), not this run"),
+    "C3": (1.0150 * 128 * 2 * 2048 * 8192 * 2, "scaled from the C2 capture by activated weight bytes, not this run"),
+    "HOTPROBE": (1.88e9, "profiles/expert_ffn_kernel_hot_probe.md (ncu, one launch), not this run"),
+}
 
 
 def measured_peaks():
@@ -70,7 +81,7 @@ def ffn_flops(p: S.Problem, counts: np.ndarray) -> float:
 
 
 class ClockSampler:
-    """SM clock and throttle reasons sampled through NVML (read-only) every 2 ms on a thread
+    """SM clock and throttle reasons sampled through NVML (read-only) every millisecond on a thread
     while the timed region runs."""
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
@@ -97,7 +108,7 @@ class ClockSampler:
                     except Exception as e:   # keep the bench alive; report what happened
                         self.err = repr(e)
                         return
-                    time.sleep(0.002)
+                    time.sleep(0.001)
             self._thread = threading.Thread(target=loop, daemon=True)
             self._thread.start()
         except Exception as e:
@@ -219,11 +230,9 @@ def workload_config(w):
             "parallelism": "independent replicas, one per GPU, no data-path collective"}
 
 
-def run_ours(args, w):
+def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline):
+    """All measurements of one workload on this rank's GPU; returns the result record (rank 0) or None."""
     from paper_2405_18832_b200 import binding as B
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-    dist, rank, world, local = dist_setup("nccl")
-    dev = torch.device("cuda", local)
     p = w.problem
     w = replica_workload(w, rank, world)
     g = generate_inputs(w, dev)
@@ -232,6 +241,7 @@ def run_ours(args, w):
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)      # four times the 126 MB L2
     stream = torch.cuda.current_stream()
     L = B.lib()
+    warmup = max(args.warmup, 3)
 
     fuse = bool(args.fuse_combine) and p.top_k == 1 and p.dtype == "bf16"
 
@@ -263,7 +273,7 @@ def run_ours(args, w):
         if ev is not None:
             ev[4].record(stream)
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(warmup):
         flush.fill_(1)
         layer()
     B.monde_poll_device_status(buf.ws)
@@ -273,7 +283,7 @@ def run_ours(args, w):
     # ---- timed region: device-resident inputs --------------------------------------
     # Events bracket whole steps only: the four calls overlap through programmatic dependent
     # launch, and an event recorded between two calls would serialise them.
-    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
@@ -292,22 +302,22 @@ def run_ours(args, w):
     launches = L.monde_kernel_launches() - launches0
     if dist is not None:
         dist.barrier()
-    clocks = sampler.stop()
-    sys.setswitchinterval(switch_interval)
     B.monde_poll_device_status(buf.ws)
     step_ms = [a.elapsed_time(b) for a, b in events]
     total_ms = max_over_ranks(dist, sum(step_ms), dev)
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / steps
     value = aggregate_tokens_per_s(p.T, world, ms_per_step)
 
     # ---- per-call pass: the same K steps again with an event between the calls, which gives
     # each call's own duration (and the dominant kernel's, for the roofline) at the price of
-    # the overlap between calls.
-    call_events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    # the overlap between calls.  The clock sampler keeps running: same load, more samples.
+    call_events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
     for ev in call_events:
         flush.fill_(2)
         layer(ev)
     torch.cuda.synchronize()
+    clocks = sampler.stop()
+    sys.setswitchinterval(switch_interval)
     call_ms = [[e[i].elapsed_time(e[i + 1]) for e in call_events] for i in range(4)]
 
     # ---- end to end: tokens in pinned host memory ----------------------------------
@@ -320,7 +330,7 @@ def run_ours(args, w):
     out_host = torch.empty((p.T, p.d_model), dtype=p.torch_dtype).pin_memory()
     for _ in range(3):
         B.moe_ffn_layer_forward_host(p, x_host, out_host, d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"], buf)
-    e2e_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    e2e_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     torch.cuda.synchronize()
     for a, b in e2e_ev:
         flush.fill_(3)
@@ -329,13 +339,13 @@ def run_ours(args, w):
         b.record(stream)
     torch.cuda.synchronize()
     serial_ms = max_over_ranks(dist, sum(a.elapsed_time(b) for a, b in e2e_ev), dev)
-    e2e_serial_value = aggregate_tokens_per_s(p.T, world, serial_ms / args.steps)
+    e2e_serial_value = aggregate_tokens_per_s(p.T, world, serial_ms / steps)
     assert torch.equal(out_host, buf.out.cpu())
 
     pipe = B.HostPipeline(p, depth=2, device=dev)
     weights = (d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"])
     out_host.zero_()
-    for _ in range(max(3, args.warmup)):
+    for _ in range(warmup):
         pipe.submit(x_host, out_host, *weights)
     pipe.wait()
     torch.cuda.synchronize()
@@ -343,48 +353,58 @@ def run_ours(args, w):
     if dist is not None:
         dist.barrier()
     p_start.record(pipe.s_in)
-    for _ in range(args.steps):
+    for _ in range(steps):
         pipe.submit(x_host, out_host, *weights)
     p_end.record(pipe.s_out)
     pipe.wait()
     torch.cuda.synchronize()
     e2e_ms = max_over_ranks(dist, p_start.elapsed_time(p_end), dev)
-    e2e_value = aggregate_tokens_per_s(p.T, world, e2e_ms / args.steps)
+    e2e_value = aggregate_tokens_per_s(p.T, world, e2e_ms / steps)
     assert torch.equal(out_host, buf.out.cpu())
+    del pipe, flush
 
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
+        return None
 
     peaks = measured_peaks()
     ffn_ms = statistics.mean(call_ms[2])
     bytes_ffn = ffn_algorithmic_bytes(p, counts)
     achieved = bytes_ffn / (ffn_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "monde_moe_ffn_fwd (hot + cold expert FFN)", "achieved": achieved,
-                "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
-                "algorithmic_bytes": bytes_ffn, "ms": ffn_ms,
-                "timing": "CUDA events around the call on its stream, per-call pass of the same K steps",
-                "tflops": ffn_flops(p, counts) / (ffn_ms * 1e-3) / 1e12,
-                "tensor_frac_of_measured_burst": ffn_flops(p, counts) / (ffn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+    tflops = ffn_flops(p, counts) / (ffn_ms * 1e-3) / 1e12
+    traffic, traffic_source = NCU_TRAFFIC.get(w.name, (None, "no capture for this workload"))
+    tensor_bound = w.name == "HOTPROBE"      # the one workload whose experts sit far above the ridge
+    common = {"kernel": "expert_ffn_kernel via monde_moe_ffn_fwd (hot + cold expert FFN, both layers)",
+              "peak_source": peaks["source"], "traffic": traffic, "traffic_source": traffic_source,
+              "algorithmic_bytes": bytes_ffn, "algorithmic_flops": ffn_flops(p, counts), "ms": ffn_ms,
+              "units_per_launch": int((counts > 0).sum()), "unit": "GB/s",
+              "timing": "CUDA events around the call on its stream, per-call pass of the same K steps",
+              "hbm_gbs": achieved, "hbm_frac_of_measured": achieved / peaks["hbm_gbs"],
+              "hbm_frac_of_nominal_8000": achieved / 8000.0,
+              "tflops": tflops, "tensor_frac_of_measured_burst": tflops / peaks["bf16_tflops"],
+              "tensor_frac_of_nominal_2250": tflops / 2250.0}
+    if tensor_bound:
+        roofline = dict(common, bound="tensor", achieved=tflops, peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                        frac=tflops / peaks["bf16_tflops"])
+    else:
+        roofline = dict(common, bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], frac=achieved / peaks["hbm_gbs"])
     elementwise_bytes = (2 * p.A + 2 * p.T) * p.d_model * p.elem_bytes + p.T * p.d_model * p.elem_bytes
     layer_floor_ms = (bytes_ffn + elementwise_bytes) / (peaks["hbm_gbs"] * 1e9) * 1e3
 
-    def layer_lower_bound_ms(tflops, gbs):
+    def layer_lower_bound_ms(tflops_peak, gbs):
         # per activated expert the slower of its flops at the tensor peak and its bytes at the HBM peak,
         # plus the elementwise stages' bytes (router input, gather, combine)
         m = counts[counts > 0].astype(np.float64)
         flops_e = 4.0 * m * p.d_model * p.d_ff
         bytes_e = 2.0 * p.d_model * p.d_ff * p.elem_bytes + m * (2.0 * p.d_model + 2.0 * p.d_ff) * p.elem_bytes
-        return (np.maximum(flops_e / (tflops * 1e12), bytes_e / (gbs * 1e9)).sum() + elementwise_bytes / (gbs * 1e9)) * 1e3
+        return (np.maximum(flops_e / (tflops_peak * 1e12), bytes_e / (gbs * 1e9)).sum()
+                + elementwise_bytes / (gbs * 1e9)) * 1e3
 
     lb_measured = layer_lower_bound_ms(peaks["bf16_tflops"], peaks["hbm_gbs"])
     lb_nominal = layer_lower_bound_ms(2250.0, 8000.0)
 
     # ---- CPU baseline: the oracle as it stands, on a bounded sample ------------------
     cpu = None
-    if not args.no_cpu_baseline and world == 1:
+    if with_cpu_baseline and world == 1:
         import oracle
         host = host_inputs(g)
         n_tok = pick_sample_tokens(w, host, 12.0)
@@ -394,16 +414,17 @@ def run_ours(args, w):
         cpu = {"value": n_tok / sec, "unit": UNIT, "cores": oracle.usable_cores(), "kind": "oracle",
                "sample": f"whole layer on the first {n_tok} of {p.T} tokens, {sec:.1f} s",
                "one_thread": {"value": n_one / sec_one, "sample": f"first {n_one} tokens, {sec_one:.1f} s"}}
+        del host
 
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+    return {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": p.dtype, "data": "synthetic", "config": workload_config(w),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
                 "d2h_bytes_per_step": out_host.numel() * out_host.element_size(),
                 "mode": "pipelined over 3 streams, 2 buffer sets: every step does its own H2D, 4 calls and D2H",
-                "serial_value": e2e_serial_value, "ms_per_step": e2e_ms / args.steps},
+                "serial_value": e2e_serial_value, "ms_per_step": e2e_ms / steps},
         "gpu_launches": launches,
         "roofline": roofline, "cpu_baseline": cpu,
         "calls_ms": {"route": statistics.mean(call_ms[0]), "permute": statistics.mean(call_ms[1]),
@@ -422,7 +443,36 @@ def run_ours(args, w):
                     "max_count": int(counts.max()), "assignments": int(counts.sum())},
         "wall_s_timed_region": wall,
     }
-    print(json.dumps(line))
+
+
+SUB_WORKLOADS = ("C2", "C1", "HOTPROBE")
+SUB_KEYS = ("value", "unit", "steps", "ms_per_step", "config", "clocks", "e2e", "roofline", "calls_ms", "calls_ms_sum",
+            "layer_lower_bound", "layer_roofline_frac", "step_ms", "routing", "gpu_launches")
+
+
+def sub_steps(name: str, steps: int) -> int:
+    """Steps of a sub-workload: at least the headline's K, and enough of them that the timed region
+    spans some 40 ms, so that the clock record has a dozen samples even for a 0.1 ms step."""
+    floor_ms = {"C1": 0.16, "C2": 0.11, "HOTPROBE": 1.0}.get(name, 1.0)
+    return max(steps, int(40.0 / floor_ms))
+
+
+def run_ours(args, w):
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    dist, rank, world, local = dist_setup("nccl")
+    dev = torch.device("cuda", local)
+    line = measure(args, w, dist, rank, world, dev, args.steps, not args.no_cpu_baseline)
+    if not args.no_sub_workloads and w.name == "C3":
+        per = {}
+        for name in SUB_WORKLOADS:
+            torch.cuda.empty_cache()
+            rec = measure(args, S.config(name), dist, rank, world, dev, sub_steps(name, args.steps), False)
+            if rec is not None:
+                per[name] = {k: rec[k] for k in SUB_KEYS}
+        if line is not None:
+            line["per_workload"] = per
+    if line is not None:
+        print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
 
@@ -430,12 +480,15 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="C1",
-                    help="C1 (default), C2, C3, or a crossover-sweep point C4:<d_model>:<T>:<zipf alpha>:<threshold>")
+    ap.add_argument("--workload", default="C3",
+                    help="C3 (default, with C2 / C1 / HOTPROBE as sub-records), C2, C1, HOTPROBE, or a crossover-sweep "
+                         "point C4:<d_model>:<T>:<zipf alpha>:<threshold>")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sub-workloads", action="store_true",
+                    help="headline workload only (no per_workload records for C2, C1 and the hot-tiling probe)")
     ap.add_argument("--fuse-combine", action="store_true",
                     help="top-1 workloads: monde_moe_ffn_combine_fwd instead of monde_moe_ffn_fwd + monde_combine")
     ap.add_argument("--policy", default="threshold", choices=["threshold", "top_h"],

@@ -14,7 +14,10 @@
  *
  * Conventions for every call
  *  - All tensor pointers are DEVICE pointers owned by the caller.  The library
- *    allocates and frees no device memory and keeps no state between calls.
+ *    allocates and frees no device memory.  Between calls it keeps nothing that a result
+ *    depends on: only which devices have had their one-time kernel set-up, and a small
+ *    cache of TMA descriptors keyed by address and shape (both under a mutex).  The
+ *    switches of monde_diagnostics.h are process-wide state and off by default.
  *  - Tensors are row-major with the last index contiguous; base pointers are
  *    16-byte aligned (cudaMalloc-style 256-byte alignment recommended).
  *  - `stream` is a cudaStream_t cast to void* (NULL = the legacy default stream).
@@ -210,8 +213,9 @@ int monde_poll_device_status(void* ws, void* stream, int32_t* site);
  *    launches.  Two calls that overlap on the GPU - different streams, or the same stream
  *    from two threads without ordering - race on the array and give undefined results:
  *    order them, or use monde_moe_ffn_fwd with separate workspaces.
- *  - After MONDE_ERR_TIMEOUT from a previous call nothing special is needed: the next call
- *    clears the header again.  monde_poll_device_status does not apply (no caller-visible ws).
+ *  - Errors found on the device (a bounded wait that ran out) are recorded in the array's
+ *    header.  The next call clears the header again, so a caller that wants to know must ask
+ *    before it: monde_poll_static_ws_status.
  */
 #define MONDE_STATIC_WS_BYTES (32u << 20)
 int monde_moe_ffn_fwd_static_ws(const monde_problem* p, const void* x_perm,
@@ -219,6 +223,14 @@ int monde_moe_ffn_fwd_static_ws(const monde_problem* p, const void* x_perm,
                                 const int32_t* counts, const int32_t* offsets, const uint8_t* cls,
                                 const int32_t* hot_ids, const int32_t* cold_ids, const int32_t* n_hot_cold,
                                 void* y_perm, void* stream);
+
+/* monde_poll_device_status for the built-in scratch array of monde_moe_ffn_fwd_static_ws (the
+ * paper has no counterpart): synchronises `stream`, then returns and clears the status word that
+ * the kernels of the last static-workspace call on the current device left in the array
+ * (MONDE_OK, or MONDE_ERR_TIMEOUT with `site` as above; y_perm of that call is then undefined).
+ * Allocates nothing.  Call it after the call it is asked about and before the next
+ * static-workspace call on that GPU, which clears the word. */
+int monde_poll_static_ws_status(void* stream, int32_t* site);
 
 /* Diagnostic: number of kernels this library has launched in this process so far. */
 long long monde_kernel_launches(void);

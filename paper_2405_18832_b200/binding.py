@@ -18,7 +18,9 @@ LIB_PATH = os.path.join(_HERE, "libmonde.so")
 
 SYMBOLS = ("monde_workspace_bytes", "monde_status_string", "monde_route", "monde_classify_top_h", "monde_permute",
            "monde_moe_ffn_fwd", "monde_moe_ffn_combine_fwd", "monde_moe_ffn_fwd_static_ws", "monde_combine", "monde_poll_device_status",
-           "monde_kernel_launches")
+           "monde_kernel_launches", "monde_poll_static_ws_status",
+           "monde_diag_set_ffn_cta_pairs", "monde_diag_set_trace", "monde_diag_set_wait_limit_ns",
+           "monde_diag_set_hold_hidden_ready", "monde_diag_device_setups")
 
 _DTYPE = {"f32": 0, "bf16": 1}
 _ACT = {"relu": 0, "gelu": 1}
@@ -75,6 +77,18 @@ def lib() -> ctypes.CDLL:
         L.monde_poll_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.monde_kernel_launches.restype = ctypes.c_longlong
         L.monde_kernel_launches.argtypes = []
+        L.monde_poll_static_ws_status.restype = ctypes.c_int
+        L.monde_poll_static_ws_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
+        L.monde_diag_set_ffn_cta_pairs.restype = None
+        L.monde_diag_set_ffn_cta_pairs.argtypes = [ctypes.c_int]
+        L.monde_diag_set_trace.restype = None
+        L.monde_diag_set_trace.argtypes = [vp, ctypes.c_int]
+        L.monde_diag_set_wait_limit_ns.restype = None
+        L.monde_diag_set_wait_limit_ns.argtypes = [ctypes.c_ulonglong]
+        L.monde_diag_set_hold_hidden_ready.restype = None
+        L.monde_diag_set_hold_hidden_ready.argtypes = [ctypes.c_int]
+        L.monde_diag_device_setups.restype = ctypes.c_int
+        L.monde_diag_device_setups.argtypes = [ctypes.c_int]
         _lib = L
     return _lib
 
@@ -164,6 +178,16 @@ def monde_moe_ffn_fwd_static_ws(p, x_perm, W1, b1, W2, b2, counts, offsets, cls,
     _check("monde_moe_ffn_fwd_static_ws", lib().monde_moe_ffn_fwd_static_ws(
         ctypes.byref(cp), _ptr(x_perm), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(counts), _ptr(offsets),
         _ptr(cls), _ptr(hot_ids), _ptr(cold_ids), _ptr(n_hot_cold), _ptr(y_perm), _stream(stream)))
+
+
+def monde_poll_static_ws_status(stream=None) -> None:
+    """monde_poll_device_status for the built-in scratch of monde_moe_ffn_fwd_static_ws: synchronises
+    the stream and raises if the last static-workspace call on this GPU recorded a device-side error.
+    Ask before the next static-workspace call, which clears the record."""
+    site = ctypes.c_int32(0)
+    st = lib().monde_poll_static_ws_status(_stream(stream), ctypes.byref(site))
+    if st != 0:
+        raise MondeError(f"device status of the static workspace (site {site.value})", st)
 
 
 def monde_combine(p, y_perm, inv_perm, topk_w, out, stream=None) -> None:

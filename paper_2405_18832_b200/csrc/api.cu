@@ -1,8 +1,8 @@
 // extern "C" entry points: argument checks, workspace carving, launches.
 #include <atomic>
-#include <cstdlib>
-#include <cstring>
+#include <mutex>
 
+#include "../../include/monde_diagnostics.h"
 #include "common.cuh"
 
 namespace monde {
@@ -23,6 +23,60 @@ int check_problem(const monde_problem* p) {
 static std::atomic<long long> g_launches{0};
 void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+// ---- per-device set-up bookkeeping ----------------------------------------------------------
+namespace {
+std::mutex g_dev_mutex;
+// 0: not run on that device yet; 1: ran and succeeded; otherwise 2 + the cudaError_t it returned
+int g_setup[kMaxDevices][kSetupKeys] = {};
+int g_sms[kMaxDevices] = {};
+}  // namespace
+
+cudaError_t per_device_once(int key, cudaError_t (*fn)()) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices || key < 0 || key >= kSetupKeys) return cudaErrorInvalidValue;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    int& state = g_setup[dev][key];
+    if (state == 0) {
+        e = fn();
+        state = e == cudaSuccess ? 1 : 2 + static_cast<int>(e);
+    }
+    return state == 1 ? cudaSuccess : static_cast<cudaError_t>(state - 2);
+}
+
+int current_sm_count() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (g_sms[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        g_sms[dev] = v;
+    }
+    return g_sms[dev];
+}
+
+// ---- diagnostic switches --------------------------------------------------------------------
+namespace {
+constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;   // 2 s
+std::atomic<unsigned long long*> g_trace{nullptr};
+std::atomic<int> g_trace_slots{0};
+std::atomic<int> g_ffn_pair{-1};
+std::atomic<unsigned long long> g_wait_limit_ns{kDefaultWaitLimitNs};
+std::atomic<int> g_hold_hidden_ready{0};
+}  // namespace
+
+DiagState diag_state() {
+    DiagState d;
+    d.trace = g_trace.load(std::memory_order_relaxed);
+    d.trace_slots = g_trace_slots.load(std::memory_order_relaxed);
+    d.ffn_pair = g_ffn_pair.load(std::memory_order_relaxed);
+    d.wait_limit_ns = g_wait_limit_ns.load(std::memory_order_relaxed);
+    d.hold_hidden_ready = g_hold_hidden_ready.load(std::memory_order_relaxed);
+    return d;
+}
+
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -41,15 +95,19 @@ int check_ws(const monde_problem& p, const void* ws, size_t ws_bytes) {
     return MONDE_OK;
 }
 
-bool force_simt() {
-    static const bool v = [] {
-        const char* e = std::getenv("MONDE_FFN_IMPL");
-        return e != nullptr && std::strcmp(e, "simt") == 0;
-    }();
-    return v;
+}  // namespace
+
+int check_ffn_fwd_args(const void* x_perm, const void* W1, const void* b1, const void* W2, const void* b2,
+                       const int32_t* counts, const int32_t* offsets, const uint8_t* cls, const int32_t* hot_ids,
+                       const int32_t* cold_ids, const int32_t* n_hot_cold, const void* y_perm) {
+    if (!x_perm || !W1 || !W2 || !counts || !offsets || !cls || !hot_ids || !cold_ids || !n_hot_cold || !y_perm)
+        return MONDE_ERR_INVALID_ARG;
+    if (!aligned16(x_perm) || !aligned16(W1) || !aligned16(W2) || !aligned16(y_perm) || !aligned16(b1) ||
+        !aligned16(b2))
+        return MONDE_ERR_INVALID_ARG;
+    return check_arch();
 }
 
-}  // namespace
 }  // namespace monde
 
 using namespace monde;
@@ -126,16 +184,13 @@ int monde_moe_ffn_fwd(const monde_problem* p, const void* x_perm,
     int st = check_problem(p);
     if (st != MONDE_OK) return st;
     if (p->T == 0) return MONDE_OK;
-    if (!x_perm || !W1 || !W2 || !counts || !offsets || !cls || !hot_ids || !cold_ids || !n_hot_cold || !y_perm)
-        return MONDE_ERR_INVALID_ARG;
-    if (!aligned16(x_perm) || !aligned16(W1) || !aligned16(W2) || !aligned16(y_perm) || !aligned16(b1) ||
-        !aligned16(b2))
-        return MONDE_ERR_INVALID_ARG;
+    if ((st = check_ffn_fwd_args(x_perm, W1, b1, W2, b2, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold,
+                                 y_perm)) != MONDE_OK)
+        return st;
     if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
-    if ((st = check_arch()) != MONDE_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     void* h = static_cast<char*>(ws) + WsLayout::kHidden;
-    if (p->dtype == MONDE_F32 || force_simt()) {
+    if (p->dtype == MONDE_F32) {
         // Same kernel for both classes; the class lists still select the experts.
         const int32_t* lists[2] = {hot_ids, cold_ids};
         for (int c = 0; c < 2; ++c) {
@@ -159,7 +214,7 @@ int monde_moe_ffn_combine_fwd(const monde_problem* p, const void* x_perm,
                               void* ws, size_t ws_bytes, void* stream) {
     int st = check_problem(p);
     if (st != MONDE_OK) return st;
-    if (p->top_k != 1 || p->dtype != MONDE_BF16 || force_simt()) return MONDE_ERR_UNSUPPORTED;
+    if (p->top_k != 1 || p->dtype != MONDE_BF16) return MONDE_ERR_UNSUPPORTED;
     if (p->T == 0) return MONDE_OK;
     if (!x_perm || !W1 || !W2 || !counts || !offsets || !cls || !perm || !topk_w || !out) return MONDE_ERR_INVALID_ARG;
     if (!aligned16(x_perm) || !aligned16(W1) || !aligned16(W2) || !aligned16(out) || !aligned16(b1) || !aligned16(b2))
@@ -198,6 +253,28 @@ int monde_poll_device_status(void* ws, void* stream, int32_t* site) {
         if (cudaStreamSynchronize(s) != cudaSuccess) return MONDE_ERR_CUDA;
     }
     return word[0];
+}
+
+// ---- include/monde_diagnostics.h --------------------------------------------------------------
+void monde_diag_set_ffn_cta_pairs(int mode) { g_ffn_pair.store(mode < 0 ? -1 : (mode != 0), std::memory_order_relaxed); }
+
+void monde_diag_set_trace(void* device_buf, int slots) {
+    g_trace_slots.store(device_buf != nullptr && slots > 0 ? slots : 0, std::memory_order_relaxed);
+    g_trace.store(slots > 0 ? static_cast<unsigned long long*>(device_buf) : nullptr, std::memory_order_relaxed);
+}
+
+void monde_diag_set_wait_limit_ns(unsigned long long ns) {
+    g_wait_limit_ns.store(ns == 0 ? kDefaultWaitLimitNs : ns, std::memory_order_relaxed);
+}
+
+void monde_diag_set_hold_hidden_ready(int on) { g_hold_hidden_ready.store(on != 0, std::memory_order_relaxed); }
+
+int monde_diag_device_setups(int device) {
+    if (device < 0 || device >= kMaxDevices) return -1;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    int n = 0;
+    for (int k = 0; k < kSetupKeys; ++k) n += g_setup[device][k] != 0;
+    return n;
 }
 
 }  // extern "C"

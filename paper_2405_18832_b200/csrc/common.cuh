@@ -76,6 +76,10 @@ inline WsLayout ws_layout(const monde_problem& p) {
 
 // MONDE_OK when the problem is inside the stated limits.
 int check_problem(const monde_problem* p);
+// Pointer, alignment and architecture checks of monde_moe_ffn_fwd (everything but the workspace).
+int check_ffn_fwd_args(const void* x_perm, const void* W1, const void* b1, const void* W2, const void* b2,
+                       const int32_t* counts, const int32_t* offsets, const uint8_t* cls, const int32_t* hot_ids,
+                       const int32_t* cold_ids, const int32_t* n_hot_cold, const void* y_perm);
 
 // ---- element helpers --------------------------------------------------------
 __device__ __forceinline__ float to_float(float v) { return v; }
@@ -155,6 +159,27 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
 
 // Process-wide count of kernels this library has launched (diagnostic).
 void count_launches(int n);
+
+// ---- per-device set-up ---------------------------------------------------------------------
+// Function attributes (the opt-in to more than 48 KB of dynamic shared memory) and the SM count
+// belong to a device, not to the process: a process that drives several GPUs must set them up on
+// each.  `per_device_once(key, fn)` runs `fn` once for the current device and the given key and
+// returns its (cached) result on every later call; keys are small integers owned by the callers.
+constexpr int kMaxDevices = 64;
+enum SetupKey { kSetupFfn = 0, kSetupRoute1, kSetupRoute2, kSetupRoute4, kSetupRoute8, kSetupKeys };
+cudaError_t per_device_once(int key, cudaError_t (*fn)());
+int current_sm_count();        // multiprocessors of the current device (cached per device)
+
+// ---- diagnostic switches (include/monde_diagnostics.h) ---------------------------------------
+// Process-wide, read at launch time; defaults leave the product path unchanged.
+struct DiagState {
+    unsigned long long* trace;      // per-unit device timeline of the expert FFN (null = off)
+    int trace_slots;
+    int ffn_pair;                   // -1 default, 0 single CTAs, 1 CTA pairs
+    unsigned long long wait_limit_ns;   // bound of every device-side wait
+    int hold_hidden_ready;          // 1: first-layer units do not publish their rows (a dependency wait then runs out)
+};
+DiagState diag_state();
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? MONDE_OK : MONDE_ERR_CUDA; }
 

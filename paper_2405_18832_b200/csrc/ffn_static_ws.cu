@@ -22,7 +22,7 @@ constexpr size_t kStaticWsBytes = MONDE_STATIC_WS_BYTES;
 // it is not a device address and must never be passed to a kernel or a memset.
 static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 
-constexpr int kMaxDevices = 64;
+using monde::kMaxDevices;
 std::mutex g_mutex;
 void* g_ws_ptr[kMaxDevices] = {};
 
@@ -33,7 +33,10 @@ int static_ws_ptr(void** out) {
     std::lock_guard<std::mutex> lock(g_mutex);
     if (g_ws_ptr[dev] == nullptr) {
         void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || p == nullptr) return MONDE_ERR_CUDA;
+        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();      // do not leave the failure behind for an unrelated later call to find
+            return MONDE_ERR_CUDA;
+        }
         g_ws_ptr[dev] = p;
     }
     *out = g_ws_ptr[dev];
@@ -52,6 +55,10 @@ extern "C" int monde_moe_ffn_fwd_static_ws(const monde_problem* p, const void* x
     if (p->T == 0) return MONDE_OK;
     const monde::WsLayout L = monde::ws_layout(*p);
     if (L.total > kStaticWsBytes) return MONDE_ERR_WORKSPACE;   // needs more scratch than the built-in array holds
+    // every check that can reject the call comes before the shared array is touched
+    if ((st = monde::check_ffn_fwd_args(x_perm, W1, b1, W2, b2, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold,
+                                        y_perm)) != MONDE_OK)
+        return st;
     void* ws = nullptr;
     if ((st = static_ws_ptr(&ws)) != MONDE_OK) return st;
     // The array keeps whatever the previous call left.  Everything the kernels expect to find
@@ -62,4 +69,11 @@ extern "C" int monde_moe_ffn_fwd_static_ws(const monde_problem* p, const void* x
     if (cudaMemsetAsync(ws, 0, monde::WsLayout::kHidden, s) != cudaSuccess) return MONDE_ERR_CUDA;
     return monde_moe_ffn_fwd(p, x_perm, W1, b1, W2, b2, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold, y_perm,
                              ws, kStaticWsBytes, stream);
+}
+
+extern "C" int monde_poll_static_ws_status(void* stream, int32_t* site) {
+    void* ws = nullptr;
+    const int st = static_ws_ptr(&ws);
+    if (st != MONDE_OK) return st;
+    return monde_poll_device_status(ws, stream, site);   // copies two words out, clears the header if it reports: no allocation
 }

@@ -49,17 +49,12 @@
 #include <cuda.h>
 
 #include <algorithm>
-#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
 #include "sm100.cuh"
 
 namespace monde {
-
-unsigned long long* g_trace = nullptr;
-int g_trace_slots = 0;
-int g_ffn_pair = -1;     // -1: default choice, 0: single CTAs, 1: CTA pairs
 
 namespace {
 
@@ -77,12 +72,12 @@ constexpr int kHotTokTile = 256;
 constexpr int kTilesPerUnit = 2;      // a unit covers two 128-feature tiles that share one token tile
 constexpr int kTileBytes = 192 * 1024;
 constexpr int kMailSlots = 8;        // unit indices in flight from the leader of a CTA pair to the other CTA
-constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue + kMailSlots;
+constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue + kMailSlots + 1;   // + the MMA issuer's way-out barrier
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
 constexpr int kStageOutBytes = 2 * 2 * 16 * kTileRows * 2;   // per epilogue warp set: two staging buffers of 16 tokens x 128 features
 constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kQueue * 64 + kTableInts * 4 + kStageOutBytes + 16;
 constexpr int kTmemCols = 512;        // two accumulator buffers of 256 fp32 columns
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
+constexpr uint64_t kDrainLimitNs = 200000ull;      // on the way out after a wait gave up: time allowed for copies and MMAs in flight to land
 
 enum WaitSite { kSiteProducerEmpty = 1, kSiteMmaFull = 2, kSiteMmaTmemEmpty = 3, kSiteEpilogueTmemFull = 4,
                 kSiteHiddenReady = 5, kSiteDrain = 6, kSiteQueue = 7, kSitePartials = 8 };
@@ -111,6 +106,8 @@ struct FfnParams {
     __nv_bfloat16* fuse_out;     // out [T, d_model]
     unsigned long long* trace;   // diagnostic timeline (null in normal use): [cta][unit slot][8]
     int trace_slots;
+    int hold_ready;              // diagnostic: first-layer units do not publish their rows
+    unsigned long long wait_ns;  // bound of a wait for another unit's results; waits inside the CTA get twice that
 };
 
 // Diagnostic timeline: slot 0 unit id, 1-2 producer first/last issue, 3-4 MMA first full / commit,
@@ -320,6 +317,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     auto q_full = [&](int s) { return bar0 + 8u * (kRingBars + 6 + s); };
     auto q_empty = [&](int s) { return bar0 + 8u * (kRingBars + 6 + kQueue + s); };
     auto mail_bar = [&](int s) { return bar0 + 8u * (kRingBars + 6 + 2 * kQueue + s); };
+    const uint32_t way_out_bar = bar0 + 8u * (kRingBars + 6 + 2 * kQueue + kMailSlots);
+    // Waits on another unit's results (hidden rows, partial tiles) give up after wait_ns; waits on the
+    // CTA's own barriers, which can only be waiting for one of those, after twice as long, so that the
+    // wait that names the cause is the one that reports.
+    const uint64_t kDepWaitNs = P.wait_ns, kWaitLimitNs = 2 * P.wait_ns;
     volatile int* mail = reinterpret_cast<volatile int*>(tmem_slot + 4);   // [kMailSlots]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -352,6 +354,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             mbar_init(q_empty(s), 11);      // MMA issuer, 8 epilogue warps, publisher, token-tile producer
         }
         for (int s = 0; s < kMailSlots; ++s) mbar_init(mail_bar(s), 1);   // the pair leader's scheduler
+        mbar_init(way_out_bar, 1);                                        // one commit, only after a wait gave up
         fence_barrier_init();
         for (int l = 0; l < 2; ++l) {
             prefetch_tensormap(&M.w[l][0]);
@@ -536,6 +539,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             int stage = 0, cls = -1;
             Geom gm = {};
             uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
+            uint32_t filled = 0;        // bit s: stage s has been filled at least once
             bool ok = true;
             // Publishes unit number `j` of this CTA (or the end marker) to the other roles.
             auto push_unit = [&](int j, const Unit& un) -> bool {
@@ -643,11 +647,20 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         tma_load_2d(a_dst, mw, full, kb * kBlockK, w_row, pol_w);
                     }
                     fill_bits ^= 1u << stage;
+                    filled |= 1u << stage;
                     if (++stage == na) stage = 0;
                 }
                 trace_time(P, it, 2);
                 cur = nxt;
             }
+            // A CTA must not exit while bulk copies into its shared memory are outstanding.  After a
+            // normal run every fill has been consumed (the MMA issuer waited for it) and these probes
+            // answer at once; after a wait gave up, the last fills may still be in flight: wait for
+            // them, bounded by time alone.  (Pairs: the leader's barriers count both CTAs' copies and
+            // the cluster barrier in the teardown holds the other CTA until the leader is through.)
+            if (!kPair || rank == 0)
+                for (int s = 0; s < kMaxStagesA; ++s)
+                    if ((filled >> s) & 1u) mbar_wait_deadline(full_a(s), ((fill_bits >> s) & 1u) ^ 1u, kDrainLimitNs);
         }
     } else if (warp == 7) {
         // ---- token-tile producer (operand B: rows of x_perm or of the hidden activations) -------
@@ -655,7 +668,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             const uint64_t pol_x = policy_evict_last();    // token tiles are re-read by every feature tile
             int stage = 0, cls = -1;
             Geom gm = {};
-            uint32_t fill_bits = 0;
+            uint32_t fill_bits = 0, filled = 0;
             bool ok = true;
             for (int it = 0; ok; ++it) {
                 const Unit un = pop_unit(it, false);
@@ -682,7 +695,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     if (ld_acquire(flag) < ready_target) {
                         const uint64_t t0 = global_timer_ns();
                         while (ld_acquire(flag) < ready_target) {
-                            if (*abort_flag != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
+                            if (*abort_flag != 0 || global_timer_ns() - t0 > kDepWaitNs) {
                                 report_timeout(P.status, abort_flag, kSiteHiddenReady);
                                 ok = false;
                                 break;
@@ -728,9 +741,14 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                             tma_load_2d(b_dst + j * 128, mi, full, kb * kBlockK, row0 + j, pol_x);
                     }
                     fill_bits ^= 1u << stage;
+                    filled |= 1u << stage;
                     if (++stage == nb) stage = 0;
                 }
             }
+            // copies in flight into this CTA's shared memory must land before it exits (see the weight producer)
+            if (!kPair || rank == 0)
+                for (int s = 0; s < kMaxStagesB; ++s)
+                    if ((filled >> s) & 1u) mbar_wait_deadline(full_b(s), ((fill_bits >> s) & 1u) ^ 1u, kDrainLimitNs);
         }
     } else if (warp == 1) {
         // ---- MMA issuer --------------------------------------------------------------
@@ -758,6 +776,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 if (!mbar_wait(acc_empty(b), acc.parity ^ 1u, abort_flag, kWaitLimitNs) ||
                     (un.wide && !mbar_wait(acc_empty(1), acc.other_parity, abort_flag, kWaitLimitNs))) {
                     report_timeout(P.status, abort_flag, kSiteMmaTmemEmpty);
+                    ok = false;
                     break;
                 }
                 tc_fence_after_sync();
@@ -826,6 +845,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 }
                 trace_time(P, it, 4);
             }
+            // Leaving because a wait gave up (here or in another role): MMAs issued so far may still be
+            // reading shared memory and writing tensor memory.  One more commit on a barrier of its own
+            // tells when they are done; the teardown frees tensor memory only after that.
+            if ((!ok || *abort_flag != 0) && (!kPair || rank == 0)) {
+                if (kPair) umma_commit_pair(way_out_bar); else umma_commit(way_out_bar);
+                mbar_wait_deadline(way_out_bar, 0, kDrainLimitNs);
+            }
         }
     } else if (warp < 6 || warp >= 8) {
         // ---- epilogue: TMEM -> registers -> bias, activation -> shared -> global -------------
@@ -868,7 +894,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     const int32_t* flag = P.part_done + un.tile_idx;
                     const uint64_t t0 = global_timer_ns();
                     while (ld_acquire(flag) < (u_nsplit - 1) * (kPair ? 2 : 1)) {
-                        if (*abort_flag != 0 || global_timer_ns() - t0 > kWaitLimitNs) {
+                        if (*abort_flag != 0 || global_timer_ns() - t0 > kDepWaitNs) {
                             report_timeout(P.status, abort_flag, kSitePartials);
                             break;   // the sums below are wrong but every access stays in bounds
                         }
@@ -1019,6 +1045,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 if (kPair) mbar_arrive_cluster(bar0_leader + 8u * (kRingBars + 2 + acc.b));
                 else mbar_arrive(acc_empty(acc.b));
                 if (un.layer == 0) {
+                    if (P.hold_ready) continue;     // diagnostic: the rows are never announced
                     __threadfence();
                     fence_proxy_async_all();
                     atomicAdd(P.ready + un.ready_idx, 1);
@@ -1031,6 +1058,13 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     }
 
     // ---- teardown --------------------------------------------------------------------
+    if (kPair && *abort_flag != 0) {
+        // A pair that gives up: the other CTA's copies into its own shared memory are counted on the
+        // leader's barriers, which the leader may not have armed for the last of them; allow them the
+        // time any copy needs to land before either CTA leaves.
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 50000ull) { }
+    }
     tc_fence_before_sync();
     __syncthreads();
     if (kPair) cluster_sync_all();   // neither CTA leaves while the other may still signal its barriers
@@ -1089,14 +1123,62 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, ui
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-    static int n = [] {
-        int dev = 0, v = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-        return v > 0 ? v : 148;
-    }();
-    return n;
+// Opt-in to the kernel's dynamic shared memory; a per-device attribute (see per_device_once).
+cudaError_t ffn_kernel_attributes() {
+    const void* kernels[4] = {
+        reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_RELU, false>),
+        reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_GELU_ERF, false>),
+        reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_RELU, true>),
+        reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_GELU_ERF, true>)};
+    for (int i = 0; i < 4; ++i) {
+        const cudaError_t e = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+// The ten tensor maps of a call depend only on addresses and shapes, never on memory contents, and a
+// layer is called again and again with the same buffers: the last few sets are kept (per process,
+// under a mutex) so that a repeated call skips ten driver calls on its host path.
+struct MapKey {
+    int dev;
+    const void *W1, *W2, *x, *h;
+    uint64_t A;
+    int E, d_model, d_ff, pair;
+    bool operator==(const MapKey& o) const {
+        return dev == o.dev && W1 == o.W1 && W2 == o.W2 && x == o.x && h == o.h && A == o.A && E == o.E &&
+               d_model == o.d_model && d_ff == o.d_ff && pair == o.pair;
+    }
+};
+constexpr int kMapCacheSlots = 16;
+std::mutex g_map_mutex;
+MapKey g_map_keys[kMapCacheSlots];
+FfnMaps g_map_vals[kMapCacheSlots];
+bool g_map_used[kMapCacheSlots] = {};
+int g_map_next = 0;
+
+bool ffn_maps(const MapKey& k, FfnMaps* out) {
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    for (int i = 0; i < kMapCacheSlots; ++i)
+        if (g_map_used[i] && g_map_keys[i] == k) { *out = g_map_vals[i]; return true; }
+    FfnMaps M;
+    const uint32_t in_box_single[3] = {16, 64, 256}, in_box_pair[3] = {8, 32, 128};
+    const uint32_t* in_box = k.pair ? in_box_pair : in_box_single;
+    for (int i = 0; i < 2; ++i) {
+        if (!make_map(&M.w[0][i], k.W1, static_cast<uint64_t>(k.E) * k.d_ff, k.d_model, kTileRows << i)) return false;
+        if (!make_map(&M.w[1][i], k.W2, static_cast<uint64_t>(k.E) * k.d_model, k.d_ff, kTileRows << i)) return false;
+    }
+    for (int i = 0; i < 3; ++i) {
+        if (!make_map(&M.in[0][i], k.x, k.A, k.d_model, in_box[i])) return false;
+        if (!make_map(&M.in[1][i], k.h, k.A, k.d_ff, in_box[i])) return false;
+    }
+    const int slot = g_map_next;
+    g_map_next = (g_map_next + 1) % kMapCacheSlots;
+    g_map_keys[slot] = k;
+    g_map_vals[slot] = M;
+    g_map_used[slot] = true;
+    *out = M;
+    return true;
 }
 
 }  // namespace
@@ -1105,18 +1187,8 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
                     const void* W2, const void* b2, const int32_t* counts, const int32_t* offsets,
                     const uint8_t* cls, void* y_perm, void* ws, cudaStream_t s, const int32_t* fuse_perm,
                     const float* fuse_w, void* fuse_out) {
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        const void* kernels[4] = {
-            reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_RELU, false>),
-            reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_GELU_ERF, false>),
-            reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_RELU, true>),
-            reinterpret_cast<const void*>(expert_ffn_kernel<MONDE_ACT_GELU_ERF, true>)};
-        for (int i = 0; i < 4 && attr_err == cudaSuccess; ++i)
-            attr_err = cudaFuncSetAttribute(kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    });
-    if (attr_err != cudaSuccess) return MONDE_ERR_CUDA;
+    if (per_device_once(kSetupFfn, ffn_kernel_attributes) != cudaSuccess) return MONDE_ERR_CUDA;
+    const DiagState diag = diag_state();
     char* base = static_cast<char*>(ws);
     const uint64_t A = static_cast<uint64_t>(p.T) * p.top_k;
     FfnParams P;
@@ -1145,11 +1217,9 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     // the token tile) give the hot class the halved token-tile traffic of two-tile units without
     // filling all of tensor memory, so the epilogue overlaps the next unit's MMAs.  Measured, the
     // two modes are within 3 % of each other on every workload tried (the feed from L2, about
-    // 11 TB/s over all SMs, limits both), so single CTAs stay the default and pairs are opt-in:
-    // MONDE_FFN_PAIR=1 in the environment, or the internal switch below.
-    static const int pair_env = [] { const char* e = getenv("MONDE_FFN_PAIR"); return e ? atoi(e) : -1; }();
-    const int pair_choice = g_ffn_pair >= 0 ? g_ffn_pair : pair_env;
-    const bool pair = pair_choice > 0;
+    // 11 TB/s over all SMs, limits both), so single CTAs stay the default and pairs are opt-in
+    // (monde_diag_set_ffn_cta_pairs).
+    const bool pair = diag.ffn_pair > 0;
     if (pair) P.pair_mask = 0xF;
     const WsLayout L = ws_layout(p);
     P.n_split = L.n_split;
@@ -1164,21 +1234,19 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.fuse_perm = fuse_perm;
     P.fuse_w = fuse_w;
     P.fuse_out = static_cast<__nv_bfloat16*>(fuse_out);
-    P.trace = g_trace;
-    P.trace_slots = g_trace_slots;
+    P.trace = diag.trace;
+    P.trace_slots = diag.trace_slots;
+    P.hold_ready = diag.hold_hidden_ready;
+    P.wait_ns = diag.wait_limit_ns;
     FfnMaps M;
-    const uint32_t in_box_single[3] = {16, 64, 256}, in_box_pair[3] = {8, 32, 128};
-    const uint32_t* in_box = pair ? in_box_pair : in_box_single;
-    for (int i = 0; i < 2; ++i) {
-        if (!make_map(&M.w[0][i], W1, static_cast<uint64_t>(p.E) * p.d_ff, p.d_model, kTileRows << i)) return MONDE_ERR_CUDA;
-        if (!make_map(&M.w[1][i], W2, static_cast<uint64_t>(p.E) * p.d_model, p.d_ff, kTileRows << i)) return MONDE_ERR_CUDA;
-    }
-    for (int i = 0; i < 3; ++i) {
-        if (!make_map(&M.in[0][i], x_perm, A, p.d_model, in_box[i])) return MONDE_ERR_CUDA;
-        if (!make_map(&M.in[1][i], P.h, A, p.d_ff, in_box[i])) return MONDE_ERR_CUDA;
-    }
+    MapKey key;
+    if (cudaGetDevice(&key.dev) != cudaSuccess) return MONDE_ERR_CUDA;
+    key.W1 = W1; key.W2 = W2; key.x = x_perm; key.h = P.h; key.A = A;
+    key.E = p.E; key.d_model = p.d_model; key.d_ff = p.d_ff; key.pair = pair;
+    if (!ffn_maps(key, &M)) return MONDE_ERR_CUDA;
     cudaError_t err;
-    const dim3 grid(pair ? sm_count() & ~1 : sm_count());
+    const int sms = current_sm_count();
+    const dim3 grid(pair ? sms & ~1 : sms);
     if (pair && p.act == MONDE_ACT_RELU)
         err = launch_pdl_cluster(expert_ffn_kernel<MONDE_ACT_RELU, true>, grid, dim3(kThreads), kSmemBytes, 2, s, M, P);
     else if (pair)
@@ -1193,13 +1261,3 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
 
 }  // namespace monde
 
-// Diagnostic hook (not part of the public header): device buffer of 148 * slots * 8 uint64
-// that the FFN kernel fills with a per-unit timeline; pass null to switch it off.
-// Diagnostic / test hook (not part of the public header): 1 runs the expert FFN on CTA pairs
-// (tcgen05 cta_group::2), 0 on single CTAs, -1 restores the default.
-extern "C" void monde_internal_set_ffn_pair(int mode) { monde::g_ffn_pair = mode; }
-
-extern "C" void monde_internal_set_trace(void* device_buf, int slots) {
-    monde::g_trace = static_cast<unsigned long long*>(device_buf);
-    monde::g_trace_slots = slots;
-}

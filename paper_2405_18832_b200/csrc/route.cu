@@ -337,25 +337,25 @@ __global__ void __launch_bounds__(512, (kDeep || kTilesPerWarp >= 8) ? 1 : 2) ro
 }
 
 template <int kTilesPerWarp>
+cudaError_t route_mma_attributes() {
+    constexpr int kSmem = 4 * 16 * (32 * kTilesPerWarp + 1) * 4;
+    const cudaError_t e = cudaFuncSetAttribute(route_mma_kernel<kTilesPerWarp, false>,
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    return e != cudaSuccess ? e : cudaFuncSetAttribute(route_mma_kernel<kTilesPerWarp, true>,
+                                                       cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+}
+
+template <int kTilesPerWarp>
 int launch_route_mma(const monde_problem& p, const void* x, const void* Wg, const float* bg, int32_t* topk_idx,
                      float* topk_w, float* probs, const HistArgs& hist, cudaStream_t s) {
     constexpr int kSmem = 4 * 16 * (32 * kTilesPerWarp + 1) * 4;
-    if (kSmem > 48 * 1024) {
-        static const cudaError_t attr = [] {
-            cudaError_t e = cudaFuncSetAttribute(route_mma_kernel<kTilesPerWarp, false>,
-                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-            return e != cudaSuccess ? e : cudaFuncSetAttribute(route_mma_kernel<kTilesPerWarp, true>,
-                                                               cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-        }();
-        if (attr != cudaSuccess) return MONDE_ERR_CUDA;
+    if (kSmem > 48 * 1024) {      // more dynamic shared memory than the default limit: opt in, once per device
+        constexpr int key = kTilesPerWarp == 1 ? kSetupRoute1 : kTilesPerWarp == 2 ? kSetupRoute2
+                          : kTilesPerWarp == 4 ? kSetupRoute4 : kSetupRoute8;
+        if (per_device_once(key, route_mma_attributes<kTilesPerWarp>) != cudaSuccess) return MONDE_ERR_CUDA;
     }
     const int grid = (p.T + 15) / 16;
-    static const int sms = [] {
-        int dev = 0, v = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-        return v > 0 ? v : 148;
-    }();
+    const int sms = current_sm_count();
     if (grid <= sms)
         launch_pdl(route_mma_kernel<kTilesPerWarp, true>, dim3(grid), dim3(512), kSmem, s,
             p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),

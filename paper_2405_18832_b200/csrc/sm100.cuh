@@ -60,6 +60,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Wait bounded by time alone (no abort flag): used on the way out of a kernel, where a thread
+// must see the asynchronous work it started (bulk copies into shared memory, MMAs) complete
+// before the CTA may exit, whatever made it leave.
+__device__ __forceinline__ bool mbar_wait_deadline(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 0 && global_timer_ns() - t0 > limit_ns) return false;
+    }
+}
+
 // ---- TMA --------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

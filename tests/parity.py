@@ -94,6 +94,91 @@ def check_full(w: S.Workload, g=None, dev=None):
     return SimpleNamespace(buf=buf, route=r, perm=pm, y_err=y_err, out_err=out_err)
 
 
+class OracleSample:
+    """Oracle outputs for a set of rows of the expert-contiguous buffer and a set of tokens, computed once
+    and compared with any number of device runs on the same inputs (the expert outputs do not depend on
+    the hot/cold classes).  Expert weights come to the host one expert at a time, so multi-gigabyte
+    layers never need a host copy of all weights."""
+
+    def __init__(self, w: S.Workload, g, dev, route, perm, rows=None, tokens=None):
+        p = w.problem
+        self.p, self.route, self.perm = p, route, perm
+        A = p.T * p.top_k
+        self.tokens = np.arange(p.T) if tokens is None else np.asarray(tokens, np.int64)
+        need = perm.inv_perm[(self.tokens[:, None] * p.top_k + np.arange(p.top_k)[None, :]).reshape(-1)]
+        rows = np.arange(A) if rows is None else np.asarray(rows, np.int64)
+        self.rows = np.unique(np.concatenate([rows, need.astype(np.int64)]))
+        row_expert = oracle.experts_of_rows(route.offsets)[self.rows]
+        self.y_ref = np.zeros((self.rows.size, p.d_model))
+        for e in np.unique(row_expert):          # one expert's weights on the host at a time
+            sel = np.nonzero(row_expert == e)[0]
+            W1 = S.as_numpy(dev["W1"][e:e + 1]); W2 = S.as_numpy(dev["W2"][e:e + 1])
+            b1 = S.as_numpy(dev["b1"][e:e + 1]) if dev["b1"] is not None else None
+            b2 = S.as_numpy(dev["b2"][e:e + 1]) if dev["b2"] is not None else None
+            self.y_ref[sel] = oracle.expert_ffn(perm.x_perm[self.rows[sel]], np.zeros(sel.size, np.int32),
+                                                W1, b1, W2, b2, p.act)
+        # combine on the sampled tokens: their rows renumbered into the sample
+        where = np.searchsorted(self.rows, need).astype(np.int32)
+        self.out_ref = oracle.combine(self.y_ref, where, np.ascontiguousarray(route.topk_w[self.tokens]))
+        self.experts_covered = np.unique(row_expert)
+
+    def compare(self, buf, label=""):
+        p = self.p
+        y_got = widen(buf.y_perm[torch.as_tensor(self.rows, device=buf.y_perm.device)])
+        y_err = check_close(f"y_perm{label}", y_got, self.y_ref, p.dtype)
+        out_got = widen(buf.out[torch.as_tensor(self.tokens, device=buf.out.device)])
+        out_err = check_close(f"out{label}", out_got, self.out_ref, p.dtype)
+        assert torch.isfinite(buf.out.float()).all() and torch.isfinite(buf.y_perm.float()).all()
+        return y_err, out_err
+
+
+def sample_rows_by_expert(route, perm, p, n_tokens, row_budget):
+    """Rows for a sampled comparison of a layer too large for the oracle in full: one whole expert
+    from the few-token end of the histogram, one whole expert with at least 64 rows (hot at every
+    threshold of the sweep), the rows around the first 256-row tile boundary of the busiest expert,
+    and the rows of every (T / n_tokens)-th token."""
+    counts, offsets = route.counts.astype(np.int64), route.offsets.astype(np.int64)
+    active = np.nonzero(counts > 0)[0]
+    rows = []
+    least = active[np.argmin(counts[active])]
+    rows.append(np.arange(offsets[least], offsets[least + 1]))
+    big = active[counts[active] >= 64]
+    if big.size:
+        e = big[np.argmin(counts[big])]
+        rows.append(np.arange(offsets[e], offsets[e + 1]))
+    top = active[np.argmax(counts[active])]
+    if counts[top] > 256:
+        rows.append(offsets[top] + np.arange(224, min(counts[top], 304)))
+    rows = np.unique(np.concatenate(rows))[:row_budget]
+    tokens = np.arange(0, p.T, max(1, -(-p.T // n_tokens)))
+    return rows, tokens
+
+
+def check_by_expert(w: S.Workload, g, dev, thresholds=None, full_flop_limit=3.0e11, n_tokens=64, row_budget=512):
+    """Parity of a layer whose weights live on the device only.  Routing integers are bit-exact in
+    full at every threshold; expert outputs and the combined output are compared with the oracle on
+    ALL rows and tokens when the layer is at most `full_flop_limit` flop, else on whole experts plus
+    a token sample (sample_rows_by_expert).  Every threshold's device output is compared with the
+    same oracle values."""
+    import dataclasses
+    p = w.problem
+    thresholds = [p.hot_threshold] if thresholds is None else list(thresholds)
+    sample, results = None, []
+    for theta in thresholds:
+        pt = dataclasses.replace(p, hot_threshold=theta)
+        buf = run_gpu(pt, dev, want_probs=False)
+        r, pm = check_routing(pt, g, buf)
+        if sample is None:
+            if 4.0 * p.A * p.d_model * p.d_ff <= full_flop_limit:
+                sample = OracleSample(w, g, dev, r, pm)
+            else:
+                rows, tokens = sample_rows_by_expert(r, pm, p, n_tokens, row_budget)
+                sample = OracleSample(w, g, dev, r, pm, rows, tokens)
+        y_err, out_err = sample.compare(buf, f" theta={theta}")
+        results.append(SimpleNamespace(buf=buf, route=r, perm=pm, y_err=y_err, out_err=out_err, theta=theta))
+    return SimpleNamespace(sample=sample, runs=results, full=sample.rows.size == p.A)
+
+
 def check_sampled(w: S.Workload, g, dev, n_tokens=96, buf=None):
     """Full-size parity: routing in full (bit-exact), expert outputs and the combined
     output on a deterministic sample of tokens, one oracle FFN row at a time."""
@@ -119,3 +204,37 @@ def check_sampled(w: S.Workload, g, dev, n_tokens=96, buf=None):
     out_err = check_close("out(sample)", out_got, out_ref, p.dtype)
     assert torch.isfinite(buf.out.float()).all() and torch.isfinite(buf.y_perm.float()).all()
     return SimpleNamespace(buf=buf, route=r, perm=pm, y_err=y_err, out_err=out_err, n_rows=rows.size)
+
+
+GUARD_BYTES = 4096
+GUARD_PATTERN = 0xA5
+
+
+def guarded_layer_buffers(p):
+    """LayerBuffers whose every output (and the workspace) sits between two guard regions filled with a
+    pattern; returns (buf, check) where check() asserts that no guard byte changed.  Stands in for a
+    memory checker: a store past either end of an output lands in a guard."""
+    buf = B.LayerBuffers(p)
+    guards = []
+    for name in ("topk_idx", "topk_w", "counts", "offsets", "cls", "hot_ids", "cold_ids", "n_hot_cold", "perm",
+                 "inv_perm", "x_perm", "y_perm", "out", "ws"):
+        t = getattr(buf, name)
+        nbytes = t.numel() * t.element_size()
+        padded = (nbytes + 255) // 256 * 256              # keeps the rear guard off the tensor's last 16-byte vector
+        raw = torch.full((GUARD_BYTES + padded + GUARD_BYTES,), GUARD_PATTERN, dtype=torch.uint8, device=t.device)
+        body = raw[GUARD_BYTES:GUARD_BYTES + nbytes]
+        if name == "ws":
+            body.zero_()
+        else:
+            body.copy_(t.contiguous().view(-1).view(torch.uint8))   # keeps initial fills such as the -1 of the id lists
+        setattr(buf, name, body.view(t.dtype).view(t.shape))
+        guards.append((name, raw, nbytes))
+
+    def check():
+        torch.cuda.synchronize()
+        for name, raw, nbytes in guards:
+            front = raw[:GUARD_BYTES]
+            rear = raw[GUARD_BYTES + nbytes:]
+            assert bool((front == GUARD_PATTERN).all()), f"{name}: bytes before the buffer were written"
+            assert bool((rear == GUARD_PATTERN).all()), f"{name}: bytes after the buffer were written"
+    return buf, check

@@ -94,6 +94,27 @@ def test_fused_combine_entry_point_checks_its_arguments_on_the_host(L):
     assert L.monde_moe_ffn_combine_fwd(ctypes.byref(cp), a, a, z, a, z, a, a, a, a, a, a, a, 16, z) == 3       # workspace too small
 
 
+def test_diagnostic_switches_and_per_device_bookkeeping(L):
+    # nothing has been launched in this process: no device has had its one-time set-up
+    assert [L.monde_diag_device_setups(d) for d in (0, 1, 63)] == [0, 0, 0]
+    assert L.monde_diag_device_setups(-1) == -1 and L.monde_diag_device_setups(64) == -1
+    # the switches only record values; defaults come back with the documented arguments
+    L.monde_diag_set_wait_limit_ns(5_000_000)
+    L.monde_diag_set_wait_limit_ns(0)
+    L.monde_diag_set_hold_hidden_ready(1)
+    L.monde_diag_set_hold_hidden_ready(0)
+    L.monde_diag_set_ffn_cta_pairs(1)
+    L.monde_diag_set_ffn_cta_pairs(-1)
+    L.monde_diag_set_trace(None, 0)
+
+
+def test_static_workspace_poll_needs_a_device(L):
+    # without a CUDA device the array's address cannot be looked up: a CUDA error status, not a crash
+    import torch
+    if not torch.cuda.is_available():
+        assert L.monde_poll_static_ws_status(None, None) == 5
+
+
 def test_status_strings(L):
     assert L.monde_status_string(0) == b"ok"
     assert b"timed out" in L.monde_status_string(6)

@@ -69,6 +69,32 @@ def test_autotuner_picks_one_of_the_candidates():
     w2 = dataclasses.replace(w, seed=10)
     batches.append(S.generate(w2, with_weights=False)["x"].cuda())
     alpha, report = policy.autotune_alpha(w.problem, batches, d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"],
-                                          1.0, 1.0, 3.0)
+                                          1.0, 1.0, 3.0, candidates=(0, 1, 2))
     assert report["chosen_offset"] in (0, 1, 2) and alpha > 0
     assert set(report["ms"]) == {0, 1, 2} and all(v > 0 for v in report["ms"].values())
+
+
+@pytest.mark.gpu
+def test_autotuner_walks_toward_the_optimum_from_both_sides():
+    # Switch-Base-like layer, two replayed batches.  With the measured feed rates (3.9 and 7.0 TB/s) Eq. 6
+    # gives H = 2 at alpha = 0.1 and H = 45 at alpha = 2.0; the measured optimum lies between (H about 11-22).
+    # A few tuning rounds from either side must not make the layer slower and must move H inward.
+    w = S.config("C1")
+    p = w.problem
+    g = S.generate(w, weights_device="cuda")
+    d = {k: (None if v is None else v.cuda()) for k, v in g.items()}
+    batches = [d["x"], S.generate(dataclasses.replace(w, seed=w.seed + 50), with_weights=False)["x"].cuda()]
+    weights = (d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"])
+    bw_hot, bw_cold = 3.9, 7.0
+
+    def ffn_ms(alpha):      # the tuner's own measurement at offset 0
+        return policy.autotune_alpha(p, batches, *weights, alpha, bw_hot, bw_cold, candidates=(0,), reps=8)[1]["ms"][0]
+
+    for start, inward in ((2.0, -1), (0.1, +1)):
+        alpha, reports = policy.autotune_alpha_rounds(p, batches, *weights, start, bw_hot, bw_cold, rounds=4,
+                                                      candidates=(-4, -2, 0, 2, 4), reps=5)
+        h_start, h_end = reports[0]["h_before"], reports[-1]["h_after"]
+        assert (h_end - h_start) * inward >= 0, (start, h_start, h_end)
+        if start == 2.0:
+            assert h_end < h_start                       # the slope on this side is a percent per step: it must move
+        assert ffn_ms(alpha) <= ffn_ms(start) * 1.02, (start, alpha)
