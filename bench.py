@@ -230,12 +230,17 @@ def workload_config(w):
             "parallelism": "independent replicas, one per GPU, no data-path collective"}
 
 
-def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline):
-    """All measurements of one workload on this rank's GPU; returns the result record (rank 0) or None."""
+def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline, weights=None, light=False):
+    """All measurements of one workload on this rank's GPU; returns the result record (rank 0) or None.
+    `weights`: expert weights already on the device (same seed and shapes), `light`: no host-buffer runs."""
     from paper_2405_18832_b200 import binding as B
     p = w.problem
     w = replica_workload(w, rank, world)
-    g = generate_inputs(w, dev)
+    if weights is None:
+        g = generate_inputs(w, dev)
+    else:
+        g = S.generate(w, with_weights=False)
+        g.update(weights)
     d = {k: (None if v is None else v.to(dev)) for k, v in g.items()}
     buf = B.LayerBuffers(p, device=dev)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)      # four times the 126 MB L2
@@ -320,6 +325,18 @@ def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline):
     sys.setswitchinterval(switch_interval)
     call_ms = [[e[i].elapsed_time(e[i + 1]) for e in call_events] for i in range(4)]
 
+    e2e = None
+    if not light:
+        e2e = measure_host_buffers(B, p, g, d, buf, flush, stream, steps, warmup, dist, dev, world)
+    del flush
+
+    if rank != 0:
+        return None
+    return summarise(args, w, p, counts, n_hot_used, steps, warmup, world, ms_per_step, step_ms, call_ms, value, clocks,
+                     launches, wall, e2e, g, with_cpu_baseline)
+
+
+def measure_host_buffers(B, p, g, d, buf, flush, stream, steps, warmup, dist, dev, world):
     # ---- end to end: tokens in pinned host memory ----------------------------------
     # Every step copies its tokens host -> device and its result device -> host.  Serial form:
     # copy, four calls, copy, wait (per-step latency).  Pipelined form (the e2e figure): the same
@@ -361,11 +378,16 @@ def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline):
     e2e_ms = max_over_ranks(dist, p_start.elapsed_time(p_end), dev)
     e2e_value = aggregate_tokens_per_s(p.T, world, e2e_ms / steps)
     assert torch.equal(out_host, buf.out.cpu())
-    del pipe, flush
+    del pipe
+    return {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
+            "d2h_bytes_per_step": out_host.numel() * out_host.element_size(),
+            "mode": "pipelined over 3 streams, 2 buffer sets: every step does its own H2D, 4 calls and D2H",
+            "serial_value": e2e_serial_value, "ms_per_step": e2e_ms / steps}
 
-    if rank != 0:
-        return None
 
+def summarise(args, w, p, counts, n_hot_used, steps, warmup, world, ms_per_step, step_ms, call_ms, value, clocks, launches,
+              wall, e2e, g, with_cpu_baseline):
+    fuse = bool(args.fuse_combine) and p.top_k == 1 and p.dtype == "bf16"
     peaks = measured_peaks()
     ffn_ms = statistics.mean(call_ms[2])
     bytes_ffn = ffn_algorithmic_bytes(p, counts)
@@ -421,10 +443,7 @@ def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline):
         "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": p.dtype, "data": "synthetic", "config": workload_config(w),
         "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
-                "d2h_bytes_per_step": out_host.numel() * out_host.element_size(),
-                "mode": "pipelined over 3 streams, 2 buffer sets: every step does its own H2D, 4 calls and D2H",
-                "serial_value": e2e_serial_value, "ms_per_step": e2e_ms / steps},
+        "e2e": e2e,
         "gpu_launches": launches,
         "roofline": roofline, "cpu_baseline": cpu,
         "calls_ms": {"route": statistics.mean(call_ms[0]), "permute": statistics.mean(call_ms[1]),
@@ -455,6 +474,59 @@ def sub_steps(name: str, steps: int) -> int:
     spans some 40 ms, so that the clock record has a dozen samples even for a 0.1 ms step."""
     floor_ms = {"C1": 0.16, "C2": 0.11, "HOTPROBE": 1.0}.get(name, 1.0)
     return max(steps, int(40.0 / floor_ms))
+
+
+SWEEP_D = (1024, 2048, 4096)
+SWEEP_T = (1, 8, 64, 512, 4096)
+SWEEP_ALPHA = (0.0, 1.2)
+SWEEP_THETA = (4, 16, 64)
+
+
+def run_sweep(args):
+    """The crossover sweep (E=64, top-2, d_ff = 4 d_model, GELU): all 90 points, one JSON line each appended
+    to `--sweep-out`; points already in the file are skipped, so an interrupted sweep resumes."""
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    done = set()
+    if os.path.exists(args.sweep_out):
+        for ln in open(args.sweep_out):
+            try:
+                r = json.loads(ln)
+                done.add((r["d_model"], r["T"], r["zipf_alpha"], r["hot_threshold"]))
+            except Exception:
+                pass
+    os.makedirs(os.path.dirname(os.path.abspath(args.sweep_out)), exist_ok=True)
+    for d_model in SWEEP_D:
+        weights = None
+        for T in SWEEP_T:
+            for alpha in SWEEP_ALPHA:
+                for theta in SWEEP_THETA:
+                    if (d_model, T, alpha, theta) in done:
+                        continue
+                    w = S.sweep_point(d_model, T, alpha, theta)
+                    if weights is None:      # same seed and tensor ids at every point of this d_model
+                        gw = S.generate(w, weights_device=dev)
+                        weights = {k: gw[k] for k in ("W1", "W2", "b1", "b2")}
+                    steps = max(args.steps, int(20.0 / (0.08 + 3.0e-8 * T * d_model)))    # about 20 ms of timed steps at least
+                    rec = measure(args, w, None, 0, 1, dev, min(steps, 200), False, weights=weights, light=True)
+                    ro = rec["roofline"]
+                    row = {"d_model": d_model, "T": T, "zipf_alpha": alpha, "hot_threshold": theta,
+                           "active": rec["routing"]["active"], "hot": rec["routing"]["hot"],
+                           "max_count": rec["routing"]["max_count"], "steps": rec["steps"],
+                           "layer_us": rec["ms_per_step"] * 1e3, "ffn_us": ro["ms"] * 1e3,
+                           "calls_us": {k: v * 1e3 for k, v in rec["calls_ms"].items()},
+                           "ffn_hbm_frac_of_measured": ro["hbm_frac_of_measured"], "ffn_tflops": ro["tflops"],
+                           "ffn_tensor_frac_of_measured_burst": ro["tensor_frac_of_measured_burst"],
+                           "layer_lower_bound_frac_of_measured": rec["layer_lower_bound"]["frac_of_measured"],
+                           "layer_lower_bound_frac_of_nominal": rec["layer_lower_bound"]["frac_of_nominal"],
+                           "cold_kernel": "tcgen05 weight-streaming tiling (no CUDA-core FMA arm exists)",
+                           "sm_mhz": rec["clocks"]["sm_mhz"], "clock_reasons": rec["clocks"]["reasons"]}
+                    with open(args.sweep_out, "a") as f:
+                        f.write(json.dumps(row) + "\n")
+                    print(json.dumps(row), flush=True)
+                    torch.cuda.empty_cache()
+        del weights
+        torch.cuda.empty_cache()
 
 
 def run_ours(args, w):
@@ -489,6 +561,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sub-workloads", action="store_true",
                     help="headline workload only (no per_workload records for C2, C1 and the hot-tiling probe)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="run the 90-point crossover sweep (resumable) instead of a single workload")
+    ap.add_argument("--sweep-out", default=os.path.join(ROOT, "gpurun_out", "sweep_C4.jsonl"))
     ap.add_argument("--fuse-combine", action="store_true",
                     help="top-1 workloads: monde_moe_ffn_combine_fwd instead of monde_moe_ffn_fwd + monde_combine")
     ap.add_argument("--policy", default="threshold", choices=["threshold", "top_h"],
@@ -497,6 +572,9 @@ def main():
     ap.add_argument("--bw-hot", type=float, default=3.9, help="TB/s at which the hot tiling consumes weights (top_h)")
     ap.add_argument("--bw-cold", type=float, default=7.0, help="TB/s at which the cold tiling streams weights (top_h)")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.workload.startswith("C4:"):
         _, d_model, T, zipf, theta = args.workload.split(":")
         w = S.sweep_point(int(d_model), int(T), float(zipf), int(theta))
