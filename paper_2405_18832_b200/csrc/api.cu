@@ -144,9 +144,8 @@ int monde_route(const monde_problem* p, const void* x, const void* Wg, const flo
     if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
     if ((st = check_arch()) != MONDE_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int32_t* ticket = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + WsLayout::kRouteTicket);
     return launch_route(*p, x, Wg, bg, topk_idx, topk_w, probs, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold,
-                        ticket, s);
+                        ws, s);
 }
 
 int monde_classify_top_h(const monde_problem* p, const int32_t* counts, double alpha, double bw_hot_feed,
@@ -172,8 +171,7 @@ int monde_permute(const monde_problem* p, const void* x, const int32_t* topk_idx
     if (!aligned16(x) || !aligned16(x_perm)) return MONDE_ERR_INVALID_ARG;
     if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
     if ((st = check_arch()) != MONDE_OK) return st;
-    int32_t* scratch = reinterpret_cast<int32_t*>(static_cast<char*>(ws) + WsLayout::kHidden);
-    return launch_permute(*p, x, topk_idx, offsets, perm, inv_perm, x_perm, scratch, static_cast<cudaStream_t>(stream));
+    return launch_permute(*p, x, topk_idx, offsets, perm, inv_perm, x_perm, ws, static_cast<cudaStream_t>(stream));
 }
 
 int monde_moe_ffn_fwd(const monde_problem* p, const void* x_perm,

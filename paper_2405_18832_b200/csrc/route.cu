@@ -2,6 +2,15 @@
 // shared-memory histogram / hot-cold classification / scan over experts.
 // Paper: Section 2.1 (gating network, score map, top-k routing); Section 2.2 (hot and
 // cold experts by token count); Eq. 5 (activated = at least one token).
+//
+// Every router CTA owns one chunk of 16 tokens.  It leaves the chunk's per-expert assignment
+// counts in the workspace (one byte each); the CTA that finishes last adds them up over
+// super-chunks of 16 chunks, which gives the per-expert totals (the histogram) and, for the
+// permutation that follows, the number of assignments to each expert in all earlier
+// super-chunks.  No CTA ever walks the assignment list again.
+// Batches of up to 256 tokens have too few chunks to occupy the GPU: their gate GEMM is dealt
+// over (chunk, 8 experts) CTAs that exchange logits through the workspace, and the CTA that
+// completes a chunk's logits does its softmax and top-k.
 #include "common.cuh"
 
 namespace monde {
@@ -23,9 +32,11 @@ __device__ __forceinline__ float warp_max(float v) {
 
 // Softmax over all E logits and the k best of them, for one token held by one warp.
 // logit[s] of lane l is expert s*32+l (-inf beyond E).
+// `chunk_hist` (shared memory, zeroed, one int per expert) counts the picks of the CTA's 16 tokens.
 __device__ __forceinline__ void softmax_topk_store(const float (&logit)[kSlots], int E, int k, int renorm,
                                                    int64_t t, int lane, int32_t* __restrict__ topk_idx,
-                                                   float* __restrict__ topk_w, float* __restrict__ probs) {
+                                                   float* __restrict__ topk_w, float* __restrict__ probs,
+                                                   int* chunk_hist) {
     float m = -INFINITY;
 #pragma unroll
     for (int s = 0; s < kSlots; ++s) m = fmaxf(m, logit[s]);
@@ -81,51 +92,29 @@ __device__ __forceinline__ void softmax_topk_store(const float (&logit)[kSlots],
             if (j < k) {
                 topk_idx[t * k + j] = sel_e[j];
                 topk_w[t * k + j] = renorm ? sel_p[j] / mass : sel_p[j];
+                atomicAdd(&chunk_hist[sel_e[j]], 1);      // integer count in shared memory: order-free
             }
         }
     }
 }
 
 struct HistArgs {
-    int A, E, theta;
+    int T, E, theta;
+    int n_chunks, n_super;
     int32_t* counts;
     int32_t* offsets;
     uint8_t* cls;
     int32_t* hot_ids;
     int32_t* cold_ids;
     int32_t* n_hot_cold;
-    int32_t* ticket;      // CTAs of the router that have finished (left at zero)
+    int32_t* ticket;          // chunks whose routing is finished (left at zero)
+    uint8_t* chunk_counts;    // [n_chunks][E]
+    int32_t* super_before;    // [n_super][E]
 };
 
-// Histogram of assignments per expert (shared-memory atomics on integers: the sum does
-// not depend on order), then classification, compaction and exclusive scan by one warp.
-// Runs in one CTA of any size.
-__device__ void histogram_classify_scan(const HistArgs& h, const int32_t* __restrict__ topk_idx, int* hist) {
-    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) hist[e] = 0;
-    __syncthreads();
-    // The loads are batched (four 16-byte loads per thread in flight): this runs in the last CTA
-    // alone, after everything else, and one load per loop iteration would put A / blockDim.x trips
-    // to L2 on the critical path of the call.
-    const int A4 = (reinterpret_cast<uintptr_t>(topk_idx) & 15) == 0 ? h.A >> 2 : 0;
-    const int4* idx4 = reinterpret_cast<const int4*>(topk_idx);
-    for (int i = threadIdx.x; i < A4; i += 4 * blockDim.x) {
-        int4 v[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int q = i + j * blockDim.x;
-            v[j] = q < A4 ? __ldcg(idx4 + q) : make_int4(-1, -1, -1, -1);
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (v[j].x < 0) continue;
-            atomicAdd(&hist[v[j].x], 1);
-            atomicAdd(&hist[v[j].y], 1);
-            atomicAdd(&hist[v[j].z], 1);
-            atomicAdd(&hist[v[j].w], 1);
-        }
-    }
-    for (int a = A4 * 4 + threadIdx.x; a < h.A; a += blockDim.x) atomicAdd(&hist[__ldcg(topk_idx + a)], 1);
-    __syncthreads();
+// Classification, compaction and exclusive scan over the per-expert totals in hist[] (shared
+// memory); run by the first warp of one CTA.
+__device__ void classify_scan(const HistArgs& h, const int* hist) {
     if (threadIdx.x >= 32) return;
     const int lane = threadIdx.x;
     // lane owns experts [lane*8, lane*8+8)
@@ -169,39 +158,82 @@ __device__ void histogram_classify_scan(const HistArgs& h, const int32_t* __rest
     }
 }
 
-// Called by every thread of every router CTA after its top-k stores: the CTA that finishes
-// last runs the histogram, so routing is one launch.
-__device__ void finish_route(const HistArgs& h, const int32_t* topk_idx) {
+// The tail of the routing call, run by one CTA after every chunk's counts are in the workspace:
+// per super-chunk sums of the chunk counts, their exclusive scan over super-chunks (what the
+// permutation needs) and the totals (the histogram), then classification and scan.  Integer sums
+// in a fixed order: nothing depends on which CTA runs this or when.
+__device__ void histogram_classify_scan(const HistArgs& h, int* hist) {
+    const int E = h.E;
+    // 1. super_before[sc][e] <- assignments of super-chunk sc to expert e (16 byte-sized loads in flight per thread)
+    for (int i = threadIdx.x; i < h.n_super * E; i += blockDim.x) {
+        const int sc = i / E, e = i - sc * E;
+        const int c0 = sc * kSuperChunks;
+        int sum = 0;
+#pragma unroll
+        for (int c = 0; c < kSuperChunks; ++c)
+            sum += c0 + c < h.n_chunks ? static_cast<int>(__ldcg(h.chunk_counts + static_cast<size_t>(c0 + c) * E + e)) : 0;
+        h.super_before[i] = sum;
+    }
+    __syncthreads();
+    // 2. exclusive scan over super-chunks, one thread per expert (loads are independent of the running sum)
+    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) {
+        int running = 0;
+        if (e < E) {
+            for (int sc = 0; sc < h.n_super; ++sc) {
+                const int c = h.super_before[static_cast<size_t>(sc) * E + e];
+                h.super_before[static_cast<size_t>(sc) * E + e] = running;
+                running += c;
+            }
+        }
+        hist[e] = running;
+    }
+    __syncthreads();
+    classify_scan(h, hist);
+}
+
+// Called by every thread of a CTA that has finished a chunk (its top-k stores and its row of chunk
+// counts): the CTA that finishes last runs the tail, so routing is one launch.
+__device__ void finish_route(const HistArgs& h) {
     __shared__ int s_hist[kMaxExperts];
     __shared__ int s_last;
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(h.ticket, 1) == static_cast<int>(gridDim.x) - 1;
+    if (threadIdx.x == 0) s_last = atomicAdd(h.ticket, 1) == h.n_chunks - 1;
     __syncthreads();
     if (!s_last) return;
     __threadfence();
     if (threadIdx.x == 0) *h.ticket = 0;
-    histogram_classify_scan(h, topk_idx, s_hist);
+    histogram_classify_scan(h, s_hist);
+}
+
+// Writes the chunk's row of per-expert counts (called by all threads after a __syncthreads that
+// follows the last softmax_topk_store of the CTA).
+__device__ __forceinline__ void store_chunk_counts(const HistArgs& h, int chunk, const int* chunk_hist) {
+    for (int e = threadIdx.x; e < h.E; e += blockDim.x)
+        h.chunk_counts[static_cast<size_t>(chunk) * h.E + e] = static_cast<uint8_t>(chunk_hist[e]);
 }
 
 // Stand-alone form, used when there are no tokens (every count is zero).
-__global__ void __launch_bounds__(256) histogram_only_kernel(HistArgs h, const int32_t* topk_idx) {
+__global__ void __launch_bounds__(256) histogram_only_kernel(HistArgs h) {
     __shared__ int s_hist[kMaxExperts];
     pdl_launch_dependents();
     pdl_wait();
-    histogram_classify_scan(h, topk_idx, s_hist);
+    histogram_classify_scan(h, s_hist);
 }
 
-// One warp per token; lanes split d_model with 16-byte loads.
+// One warp per token (16 warps: one chunk per CTA); lanes split d_model with 16-byte loads.
 template <typename T>
-__global__ void __launch_bounds__(128) route_warp_per_token_kernel(
+__global__ void __launch_bounds__(kChunkTokens * 32) route_warp_per_token_kernel(
         int T_tokens, int d, int E, int k, int renorm, const T* __restrict__ x, const T* __restrict__ Wg,
         const float* __restrict__ bg, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
         float* __restrict__ probs, const HistArgs hist) {
     constexpr int V = Vec16<T>::N;
+    __shared__ int s_chunk[kMaxExperts];
     const int lane = threadIdx.x & 31;
-    const int64_t t = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * kChunkTokens + (threadIdx.x >> 5);
     pdl_launch_dependents();
+    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) s_chunk[e] = 0;
+    __syncthreads();
     pdl_wait();
     if (t < T_tokens) {
     const T* xr = x + t * d;
@@ -228,9 +260,11 @@ __global__ void __launch_bounds__(128) route_warp_per_token_kernel(
             }
         }
     }
-    softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs);
+    softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs, s_chunk);
     }
-    finish_route(hist, topk_idx);
+    __syncthreads();
+    store_chunk_counts(hist, blockIdx.x, s_chunk);
+    finish_route(hist);
 }
 
 // ---- bf16 gate on the warp-level tensor-core path -------------------------------------
@@ -261,11 +295,13 @@ __global__ void __launch_bounds__(512, (kDeep || kTilesPerWarp >= 8) ? 1 : 2) ro
     constexpr int kEPad = 32 * kTilesPerWarp;
     constexpr int kRow = kEPad + 1;
     extern __shared__ float s_part[];                 // [4 K quarters][16 tokens][kRow]
+    __shared__ int s_chunk[kMaxExperts];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int eq = warp & 3, kq = warp >> 2;
     const int g = lane >> 2, t4 = lane & 3;
     const int tok0 = blockIdx.x * 16;
     pdl_launch_dependents();
+    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) s_chunk[e] = 0;
     pdl_wait();
     const int r0 = min(tok0 + g, T_tokens - 1), r1 = min(tok0 + g + 8, T_tokens - 1);
     const uint4* xa = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(r0) * d) + t4;
@@ -331,9 +367,95 @@ __global__ void __launch_bounds__(512, (kDeep || kTilesPerWarp >= 8) ? 1 : 2) ro
                 logit[s] = -INFINITY;
             }
         }
-        softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs);
+        softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs, s_chunk);
     }
-    finish_route(hist, topk_idx);
+    __syncthreads();
+    store_chunk_counts(hist, blockIdx.x, s_chunk);
+    finish_route(hist);
+}
+
+// ---- small batches: the gate GEMM dealt over (chunk, 8 experts) CTAs -----------------------------
+// A batch of a few dozen tokens has one or two chunks; with one CTA per chunk a decode step would
+// read the whole gate matrix through one or two SMs.  Here CTA (chunk c, octet o) computes the
+// logits of 16 tokens against experts [8o, 8o+8): its 16 warps split K sixteen ways (all loads of
+// the CTA are in flight together: one trip to memory), partial sums meet in shared memory and are
+// added in warp order, and the 16 x 8 logits go to the workspace.  The CTA that completes a chunk's
+// logits (per-chunk ticket) runs softmax and top-k for the chunk, then the usual tail.
+__global__ void __launch_bounds__(512, 1) route_split_kernel(
+        int T_tokens, int d, int E, int k, int renorm, const __nv_bfloat16* __restrict__ x,
+        const __nv_bfloat16* __restrict__ Wg, const float* __restrict__ bg, int32_t* __restrict__ topk_idx,
+        float* __restrict__ topk_w, float* __restrict__ probs, float* __restrict__ logits_ws,
+        int32_t* __restrict__ tile_tickets, const HistArgs hist) {
+    __shared__ float s_part[16][16][9];            // [warp][token][expert of the octet]
+    __shared__ int s_chunk[kMaxExperts];
+    __shared__ int s_last;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t4 = lane & 3;
+    const int chunk = blockIdx.x, oct = blockIdx.y, n_oct = gridDim.y;
+    const int tok0 = chunk * kChunkTokens;
+    pdl_launch_dependents();
+    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) s_chunk[e] = 0;
+    pdl_wait();
+    const int r0 = min(tok0 + g, T_tokens - 1), r1 = min(tok0 + g + 8, T_tokens - 1);
+    const uint4* xa = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(r0) * d) + t4;
+    const uint4* xb = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(r1) * d) + t4;
+    const uint4* wp = reinterpret_cast<const uint4*>(Wg + static_cast<int64_t>(min(oct * 8 + g, E - 1)) * d) + t4;
+    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    const int steps = d / 32;               // 32 k per step: 4 lanes x 8 elements; warp w takes steps w, w+16, ...
+    constexpr int kBatch = 4;
+    for (int s0 = warp; s0 < steps; s0 += 16 * kBatch) {
+        uint4 a[kBatch], b[kBatch], w[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            const int sidx = s0 + 16 * i;
+            if (sidx < steps) {
+                a[i] = xa[sidx * 4];
+                b[i] = xb[sidx * 4];
+                w[i] = wp[sidx * 4];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            if (s0 + 16 * i < steps) {
+                mma_bf16_16816(acc, a[i].x, b[i].x, a[i].y, b[i].y, w[i].x, w[i].y);
+                mma_bf16_16816(acc, a[i].z, b[i].z, a[i].w, b[i].w, w[i].z, w[i].w);
+            }
+        }
+    }
+    s_part[warp][g][t4 * 2] = acc[0];
+    s_part[warp][g][t4 * 2 + 1] = acc[1];
+    s_part[warp][g + 8][t4 * 2] = acc[2];
+    s_part[warp][g + 8][t4 * 2 + 1] = acc[3];
+    __syncthreads();
+    if (threadIdx.x < 128) {               // 16 tokens x 8 experts, the 16 K slices added in warp order
+        const int tk = threadIdx.x >> 3, eo = threadIdx.x & 7;
+        float sum = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 16; ++w) sum += s_part[w][tk][eo];
+        const int e = oct * 8 + eo;
+        if (tok0 + tk < T_tokens && e < E)
+            logits_ws[static_cast<int64_t>(tok0 + tk) * kMaxExperts + e] = sum + (bg != nullptr ? bg[e] : 0.0f);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(tile_tickets + chunk, 1) == n_oct - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) tile_tickets[chunk] = 0;
+    const int64_t t = tok0 + warp;          // one warp per token for softmax and top-k
+    if (t < T_tokens) {
+        float logit[kSlots];
+#pragma unroll
+        for (int sl = 0; sl < kSlots; ++sl) {
+            const int e = sl * 32 + lane;
+            logit[sl] = e < E ? __ldcg(logits_ws + t * kMaxExperts + e) : -INFINITY;
+        }
+        softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs, s_chunk);
+    }
+    __syncthreads();
+    store_chunk_counts(hist, chunk, s_chunk);
+    finish_route(hist);
 }
 
 template <int kTilesPerWarp>
@@ -427,10 +549,23 @@ __global__ void __launch_bounds__(kMaxExperts) classify_top_h_kernel(
 
 int launch_route(const monde_problem& p, const void* x, const void* Wg, const float* bg,
                  int32_t* topk_idx, float* topk_w, float* probs, int32_t* counts, int32_t* offsets, uint8_t* cls,
-                 int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, int32_t* ticket, cudaStream_t s) {
-    const HistArgs hist{p.T * p.top_k, p.E, p.hot_threshold, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold, ticket};
+                 int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, void* ws, cudaStream_t s) {
+    const WsLayout L = ws_layout(p);
+    char* base = static_cast<char*>(ws);
+    int32_t* ticket = reinterpret_cast<int32_t*>(base + WsLayout::kRouteTicket);
+    const HistArgs hist{p.T, p.E, p.hot_threshold, L.n_chunks, L.n_super, counts, offsets, cls, hot_ids, cold_ids,
+                        n_hot_cold, ticket, reinterpret_cast<uint8_t*>(base + L.chunk_counts_off),
+                        reinterpret_cast<int32_t*>(base + L.super_before_off)};
     if (p.T == 0) {
-        launch_pdl(histogram_only_kernel, dim3(1), dim3(256), 0, s, hist, topk_idx);
+        launch_pdl(histogram_only_kernel, dim3(1), dim3(256), 0, s, hist);
+        return launched();
+    }
+    if (p.dtype == MONDE_BF16 && p.T <= kSplitRouteMaxTokens) {
+        // at most 16 chunks: their tickets follow the call's own in the workspace header
+        launch_pdl(route_split_kernel, dim3(L.n_chunks, (p.E + 7) / 8), dim3(512), 0, s,
+            p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),
+            static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs,
+            reinterpret_cast<float*>(base + L.logits_off), ticket + 1, hist);
         return launched();
     }
     if (p.dtype == MONDE_BF16) {
@@ -441,8 +576,7 @@ int launch_route(const monde_problem& p, const void* x, const void* Wg, const fl
         else st = launch_route_mma<8>(p, x, Wg, bg, topk_idx, topk_w, probs, hist, s);
         if (st != MONDE_OK) return st;
     } else {
-        const int warps = 4;
-        launch_pdl(route_warp_per_token_kernel<float>, dim3((p.T + warps - 1) / warps), dim3(warps * 32), 0, s,
+        launch_pdl(route_warp_per_token_kernel<float>, dim3(L.n_chunks), dim3(kChunkTokens * 32), 0, s,
             p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const float*>(x),
             static_cast<const float*>(Wg), bg, topk_idx, topk_w, probs, hist);
     }
