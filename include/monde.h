@@ -126,7 +126,9 @@ int monde_classify_top_h(const monde_problem* p, const int32_t* counts, double a
  * order); Section 4.1 (drop-less, padding-less routing: no capacity, no padded slot).
  *   pos(a) = offsets[e_a] + #{a' < a : e_a' = e_a};  perm[pos] = a;  inv_perm[a] = pos
  *   x_perm[pos,:] = x[a / top_k,:]
- * in : x [T,d_model]; topk_idx [T,k]; offsets [E+1]
+ * in : x [T,d_model]; topk_idx [T,k]; offsets [E+1]; and, inside `ws`, the per-chunk expert
+ *      counts that monde_route left there: call it after monde_route for the same tokens, on the
+ *      same workspace and stream
  * out: perm [A], inv_perm [A] int32; x_perm [A,d_model] (dtype)
  */
 int monde_permute(const monde_problem* p, const void* x, const int32_t* topk_idx,
@@ -166,16 +168,21 @@ int monde_moe_ffn_fwd(const monde_problem* p, const void* x_perm,
 int monde_combine(const monde_problem* p, const void* y_perm, const int32_t* inv_perm,
                   const float* topk_w, void* out, void* stream);
 
-/* Expert FFN with the combine folded into its last store, for top-1 routing (one expert per
- * token: the sum over experts has a single term, so no order of additions is lost).
+/* Expert FFN and combine in one call, without a caller-side y_perm (bf16 problems).
  * Paper: Section 2.1 (expert outputs are weighted by the gate and re-organised into the original
  * token order); Section 3.4 (kernels fuse what follows a GEMM into it, as gemm+relu does).
- *   for e with counts[e] > 0, rows r in [offsets[e], offsets[e+1]), t = perm[r]:
+ *   top_k == 1 (one expert per token: the sum over experts has a single term, so no order of
+ *   additions is lost): the FFN's last store applies the gate weight and writes `out` directly,
+ *     for rows r of expert e, t = perm[r]:
  *     out[t,:] = topk_w[t] * round_dtype(h[r,:] * W2[e]^T + b2[e])      (rounded once more to dtype)
- * i.e. bit for bit what monde_moe_ffn_fwd followed by monde_combine writes to `out`; y_perm is
- * never materialised.  Returns MONDE_ERR_UNSUPPORTED unless top_k == 1 and dtype is bf16.
+ *   top_k > 1: the FFN's last store puts every output row at its assignment id perm[r] = t*top_k + j,
+ *   so the top_k rows of a token lie side by side in a staging buffer inside the workspace, and the
+ *   combine kernel then adds them in slot order (j ascending, fp32, one rounding) with no index
+ *   look-up.
+ * Either way `out` holds bit for bit what monde_moe_ffn_fwd followed by monde_combine writes.
+ * Returns MONDE_ERR_UNSUPPORTED unless dtype is bf16.
  * in : as monde_moe_ffn_fwd (the class lists are not needed), perm [A] as written by
- *      monde_permute, topk_w [T,1] fp32
+ *      monde_permute, topk_w [T,top_k] fp32
  * out: out [T,d_model] (dtype)
  */
 int monde_moe_ffn_combine_fwd(const monde_problem* p, const void* x_perm,

@@ -158,7 +158,8 @@ def monde_moe_ffn_fwd(p, x_perm, W1, b1, W2, b2, counts, offsets, cls, hot_ids, 
 
 def monde_moe_ffn_combine_fwd(p, x_perm, W1, b1, W2, b2, counts, offsets, cls, perm, topk_w, out, ws,
                               stream=None) -> None:
-    """Expert FFN with the gate-weighted combine folded into its last store (top-1, bf16 only)."""
+    """Expert FFN and combine in one call, no y_perm (bf16 only): top-1 folds the gate weight into the FFN's
+    last store; top-k > 1 stages the rows in token order inside the workspace and adds them in slot order."""
     cp = c_problem(p)
     _check("monde_moe_ffn_combine_fwd", lib().monde_moe_ffn_combine_fwd(
         ctypes.byref(cp), _ptr(x_perm), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(counts), _ptr(offsets),
@@ -233,8 +234,8 @@ class LayerBuffers:
 def moe_ffn_layer_forward(p, x, Wg, bg, W1, b1, W2, b2, buf: LayerBuffers, stream=None,
                           fuse_combine: bool = False) -> torch.Tensor:
     """route -> permute -> expert FFN (hot + cold) -> combine, all enqueued on one stream.
-    `fuse_combine` (top-1 bf16 problems) takes the three-call form: the FFN's last store applies the
-    gate weight and writes `out` directly, same bytes, no y_perm."""
+    `fuse_combine` (bf16 problems) takes the three-call form, monde_moe_ffn_combine_fwd: same bytes in `out`,
+    no y_perm."""
     monde_route(p, x, Wg, bg, buf.topk_idx, buf.topk_w, buf.counts, buf.offsets, buf.cls, buf.hot_ids,
                 buf.cold_ids, buf.n_hot_cold, buf.probs, buf.ws, stream)
     monde_permute(p, x, buf.topk_idx, buf.offsets, buf.perm, buf.inv_perm, buf.x_perm, buf.ws, stream)

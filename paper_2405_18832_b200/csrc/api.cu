@@ -212,15 +212,23 @@ int monde_moe_ffn_combine_fwd(const monde_problem* p, const void* x_perm,
                               void* ws, size_t ws_bytes, void* stream) {
     int st = check_problem(p);
     if (st != MONDE_OK) return st;
-    if (p->top_k != 1 || p->dtype != MONDE_BF16) return MONDE_ERR_UNSUPPORTED;
+    if (p->dtype != MONDE_BF16) return MONDE_ERR_UNSUPPORTED;
     if (p->T == 0) return MONDE_OK;
     if (!x_perm || !W1 || !W2 || !counts || !offsets || !cls || !perm || !topk_w || !out) return MONDE_ERR_INVALID_ARG;
     if (!aligned16(x_perm) || !aligned16(W1) || !aligned16(W2) || !aligned16(out) || !aligned16(b1) || !aligned16(b2))
         return MONDE_ERR_INVALID_ARG;
     if ((st = check_ws(*p, ws, ws_bytes)) != MONDE_OK) return st;
     if ((st = check_arch()) != MONDE_OK) return st;
-    return launch_ffn_bf16(*p, x_perm, W1, b1, W2, b2, counts, offsets, cls, nullptr, ws,
-                           static_cast<cudaStream_t>(stream), perm, topk_w, out);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (p->top_k == 1)      // one term per token: the last store applies the gate weight and writes `out`
+        return launch_ffn_bf16(*p, x_perm, W1, b1, W2, b2, counts, offsets, cls, nullptr, ws, s, perm, topk_w, out);
+    // Several terms per token: the last store puts every expert output row at its assignment id, i.e. the
+    // top_k rows of a token side by side (a staging buffer in the workspace), and the combine kernel adds
+    // them in slot order without looking anything up: same arithmetic as monde_combine, same bytes.
+    void* stage = static_cast<char*>(ws) + ws_layout(*p).stage_off;
+    st = launch_ffn_bf16(*p, x_perm, W1, b1, W2, b2, counts, offsets, cls, nullptr, ws, s, perm, nullptr, stage);
+    if (st != MONDE_OK) return st;
+    return launch_combine(*p, stage, nullptr, topk_w, out, s);
 }
 
 int monde_combine(const monde_problem* p, const void* y_perm, const int32_t* inv_perm,

@@ -35,6 +35,7 @@ struct WsLayout {
     size_t chunk_counts_off;   // uint8 [n_chunks][E]: assignments of each 16-token chunk to each expert
     size_t super_before_off;   // int32 [n_super][E]: assignments to each expert in all earlier super-chunks
     size_t logits_off;         // fp32 [T][kMaxExperts]: gate logits of small batches, between the two phases of the split router
+    size_t stage_off;          // [T][top_k][d_model] in the problem dtype: expert outputs in token order (fused combine, top_k > 1)
     int n_chunks, n_super;
     size_t total;
 };
@@ -85,7 +86,9 @@ inline WsLayout ws_layout(const monde_problem& p) {
     l.super_before_off = round256(l.chunk_counts_off + static_cast<size_t>(l.n_chunks) * p.E);
     l.logits_off = round256(l.super_before_off + static_cast<size_t>(l.n_super) * p.E * 4);
     const size_t logits_bytes = p.T <= kSplitRouteMaxTokens ? static_cast<size_t>(p.T) * kMaxExperts * 4 : 0;
-    l.total = l.logits_off + logits_bytes + 1024;
+    l.stage_off = round256(l.logits_off + logits_bytes);
+    const size_t stage_bytes = (p.top_k > 1 && p.dtype == MONDE_BF16) ? A * p.d_model * elem_bytes(p.dtype) : 0;
+    l.total = l.stage_off + stage_bytes + 1024;
     return l;
 }
 

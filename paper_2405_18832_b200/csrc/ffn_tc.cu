@@ -101,9 +101,9 @@ struct FfnParams {
     int32_t* part_done;    // per cold second-layer tile: partial tiles finished
     float* partials;       // [tile][split][cold_tile tokens][128 features] fp32
     int32_t* ready;        // per token tile: first-layer units finished
-    const int32_t* fuse_perm;    // fused combine (top-1): assignment id of every row; null = store y
-    const float* fuse_w;         // gate weight per assignment
-    __nv_bfloat16* fuse_out;     // out [T, d_model]
+    const int32_t* fuse_perm;    // fused combine: assignment id of every row; null = store y in expert-contiguous order
+    const float* fuse_w;         // gate weight per assignment (top-1); null = rows go out unweighted, in assignment order
+    __nv_bfloat16* fuse_out;     // out [T, d_model] (top-1) or the token-ordered staging rows [T * top_k, d_model]
     unsigned long long* trace;   // diagnostic timeline (null in normal use): [cta][unit slot][8]
     int trace_slots;
     int hold_ready;              // diagnostic: first-layer units do not publish their rows
@@ -997,8 +997,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     for (int half = 0; half < 2; ++half) {
                         const int r = rd_row + half * 8;
                         if (c0 + r < u_rows) {
-                            f_tok[half] = __ldg(P.fuse_perm + u_row0 + c0 + r);     // top-1: assignment id = token id
-                            f_w[half] = __ldg(P.fuse_w + f_tok[half]);
+                            f_tok[half] = __ldg(P.fuse_perm + u_row0 + c0 + r);     // assignment id (top-1: = token id)
+                            if (P.fuse_w != nullptr) f_w[half] = __ldg(P.fuse_w + f_tok[half]);
                         }
                     }
                 }
@@ -1044,7 +1044,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                             for (int i = 0; i < 4; ++i) {
                                 const float lo = __uint_as_float(w4[i] << 16), hi = __uint_as_float(w4[i] & 0xFFFF0000u);
                                 const __nv_bfloat162 pr = __floats2bfloat162_rn(fmaf(f_w[half], lo, 0.0f), fmaf(f_w[half], hi, 0.0f));
-                                o4[i] = *reinterpret_cast<const uint32_t*>(&pr);
+                                o4[i] = P.fuse_w != nullptr ? *reinterpret_cast<const uint32_t*>(&pr) : w4[i];   // staging rows keep y as it is
                             }
                             *reinterpret_cast<uint4*>(P.fuse_out + static_cast<int64_t>(f_tok[half]) * N + n0 + rd_col) =
                                 make_uint4(o4[0], o4[1], o4[2], o4[3]);

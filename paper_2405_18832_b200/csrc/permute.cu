@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(256) combine_kernel(
 #pragma unroll
     for (int v = 0; v < V; ++v) acc[v] = 0.0f;
     for (int j = 0; j < k; ++j) {
-        const int pos = inv_perm[t * k + j];
+        const int pos = inv_perm != nullptr ? inv_perm[t * k + j] : static_cast<int>(t * k + j);   // null: rows already in token order
         const float w = topk_w[t * k + j];
         float y[V];
         Vec16<T>::load(y_perm + static_cast<int64_t>(pos) * d + c, y);

@@ -320,7 +320,7 @@ __global__ void __launch_bounds__(512, (kDeep || kTilesPerWarp >= 8) ? 1 : 2) ro
     const int steps = d / 32;               // 32 k per step: 4 lanes x 8 elements
     // Loads of several steps are issued together and the MMAs follow: a step at a time would put one
     // trip to memory per step on the critical path of a kernel that is all latency.
-    constexpr int kBatch = (!kDeep || kTilesPerWarp >= 8) ? 1 : 20 / (2 + kTilesPerWarp);   // about 80 registers of loads in flight
+    constexpr int kBatch = kTilesPerWarp >= 8 ? 1 : (kDeep ? 20 / (2 + kTilesPerWarp) : (kTilesPerWarp <= 2 ? 2 : 1));   // loads in flight: about 80 registers (deep), 32 (two CTAs per SM)
     for (int s0 = kq; s0 < steps; s0 += 4 * kBatch) {
         uint4 a[kBatch], b[kBatch], w[kBatch][kTilesPerWarp];
 #pragma unroll

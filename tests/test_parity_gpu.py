@@ -198,14 +198,27 @@ def test_host_pipeline_matches_step_by_step_results():
     assert not torch.equal(outs[0], outs[1])
 
 
-@pytest.mark.parametrize("name", ["C1", "C2", "ragged_top1"])
+FUSED_CASES = {
+    "C1": lambda: S.config("C1"),
+    "C2": lambda: S.config("C2"),
+    "ragged_top1": lambda: _wl("ragged_top1", T=777, d_model=320, d_ff=832, E=9, hot_threshold=70, zipf_alpha=1.3, act="gelu"),
+    "top2_renorm_gelu": lambda: _wl("top2", T=333, d_model=192, d_ff=448, E=12, top_k=2, renormalize=1, act="gelu",
+                                    hot_threshold=40, zipf_alpha=1.0),
+    "top4_ragged": lambda: _wl("top4", T=500, d_model=320, d_ff=832, E=10, top_k=4, renormalize=1, hot_threshold=150,
+                               zipf_alpha=1.2),
+    "C4_d1024_T512": lambda: S.sweep_point(1024, 512, 1.2, 16),
+}
+
+
+@pytest.mark.parametrize("name", list(FUSED_CASES))
 def test_fused_combine_gives_the_bytes_of_the_four_call_form(name):
-    # top-1: the FFN's last store applies the gate weight and writes `out`; must equal ffn + combine bit for bit
-    w = (_wl("ragged_top1", T=777, d_model=320, d_ff=832, E=9, hot_threshold=70, zipf_alpha=1.3, act="gelu")
-         if name == "ragged_top1" else S.config(name))
+    # top-1: the FFN's last store applies the gate weight and writes `out`; top-k: it stages the rows in token
+    # order and the combine kernel adds them without a look-up; either must equal ffn + combine bit for bit
+    w = FUSED_CASES[name]()
     p = w.problem
-    g = S.generate(w)
+    g = S.generate(w, with_weights=False)
     dev = P.to_device(g)
+    dev.update({k: v for k, v in S.generate(w, weights_device="cuda").items() if k in ("W1", "W2", "b1", "b2")})
     weights = (dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"])
     buf = B.LayerBuffers(p)
     ref = B.moe_ffn_layer_forward(p, dev["x"], *weights, buf).clone()
@@ -216,8 +229,8 @@ def test_fused_combine_gives_the_bytes_of_the_four_call_form(name):
     assert torch.equal(got, ref)
 
 
-def test_fused_combine_refuses_top2():
-    w = _wl("top2", T=64, top_k=2)
+def test_fused_combine_refuses_fp32():
+    w = S.config("C0")
     p = w.problem
     dev = P.to_device(S.generate(w))
     buf = B.LayerBuffers(p)
@@ -360,7 +373,7 @@ def test_random_shapes_on_one_shared_workspace():
             P.check_close(f"{w.name} y_perm", P.widen(buf.y_perm), y_ref, p.dtype)
             out_ref = oracle.combine(y_ref, pm.inv_perm, r.topk_w)
             P.check_close(f"{w.name} out", P.widen(buf.out), out_ref, p.dtype)
-            if p.top_k == 1:
+            if p.dtype == "bf16":
                 four_calls = buf.out.clone()
                 buf.out.zero_()
                 B.moe_ffn_layer_forward(p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"], buf,
@@ -446,7 +459,8 @@ GUARDED = [S.config("C1"), S.config("C2"),
 @pytest.mark.parametrize("w", GUARDED, ids=[w.name for w in GUARDED])
 def test_no_kernel_writes_outside_its_outputs(w, pairs):
     p = w.problem
-    dev = P.to_device(S.generate(w))
+    dev = P.to_device(S.generate(w, with_weights=False))
+    dev.update({k: v for k, v in S.generate(w, weights_device="cuda").items() if k in ("W1", "W2", "b1", "b2")})
     args = (p, dev["x"], dev["Wg"], dev["bg"], dev["W1"], dev["b1"], dev["W2"], dev["b2"])
     plain = P.run_gpu(p, dev, want_probs=False)
     B.lib().monde_diag_set_ffn_cta_pairs(pairs)
@@ -457,7 +471,7 @@ def test_no_kernel_writes_outside_its_outputs(w, pairs):
         check()
         assert torch.equal(buf.perm, plain.perm)
         P.check_close("out", P.widen(out), P.widen(plain.out), p.dtype)
-        if p.top_k == 1:
+        if p.dtype == "bf16":
             B.moe_ffn_layer_forward(*args, buf, fuse_combine=True)
             B.monde_poll_device_status(buf.ws)
             check()
@@ -467,11 +481,13 @@ def test_no_kernel_writes_outside_its_outputs(w, pairs):
 
 def test_one_time_setup_is_recorded_per_device():
     L = B.lib()
-    P.run_gpu(S.config("C2").problem, P.to_device(S.generate(S.config("C2"))), want_probs=False)
+    w = _wl("setup", T=300, d_model=256, d_ff=512, E=128, top_k=2, renormalize=1, hot_threshold=16, zipf_alpha=1.0)
+    inputs = P.to_device(S.generate(w))
+    P.run_gpu(w.problem, inputs, want_probs=False)
     dev = torch.cuda.current_device()
     n = L.monde_diag_device_setups(dev)
     assert n >= 1
-    P.run_gpu(S.config("C2").problem, P.to_device(S.generate(S.config("C2"))), want_probs=False)
+    P.run_gpu(w.problem, inputs, want_probs=False)
     assert L.monde_diag_device_setups(dev) == n                      # second call: nothing set up again
     assert L.monde_diag_device_setups(dev + 1) == 0                   # a device this process never used
     assert L.monde_diag_device_setups(64) == -1
