@@ -72,7 +72,7 @@ constexpr int kHotTokTile = 256;
 constexpr int kTilesPerUnit = 2;      // a unit covers two 128-feature tiles that share one token tile
 constexpr int kTileBytes = 192 * 1024;
 constexpr int kMailSlots = 8;        // unit indices in flight from the leader of a CTA pair to the other CTA
-constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue + kMailSlots + 1 + 2 * kMaxStagesA;   // + the MMA issuer's way-out barrier + the shared barriers of lockstep rings
+constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue + kMailSlots + 1 + 2 * kMaxStagesA + 1;   // + the MMA issuer's way-out barrier + the shared barriers of lockstep rings
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
 constexpr int kStageOutBytes = 2 * 2 * 16 * kTileRows * 2;   // per epilogue warp set: two staging buffers of 16 tokens x 128 features
 constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kQueue * 64 + kTableInts * 4 + kStageOutBytes + 16;
@@ -322,6 +322,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     // so one "full" barrier (both producers arrive on it) and one "empty" barrier (one commit) serve both.
     auto full_c = [&](int s) { return bar0 + 8u * (kRingBars + 7 + 2 * kQueue + kMailSlots + s); };
     auto empty_c = [&](int s) { return bar0 + 8u * (kRingBars + 7 + 2 * kQueue + kMailSlots + kMaxStagesA + s); };
+    // the weight producer tells the scheduler that the unit it is loading is nearly issued: time to take the next one
+    const uint32_t claim_bar = bar0 + 8u * (kRingBars + 7 + 2 * kQueue + kMailSlots + 2 * kMaxStagesA);
     // Waits on another unit's results (hidden rows, partial tiles) give up after wait_ns; waits on the
     // CTA's own barriers, which can only be waiting for one of those, after twice as long, so that the
     // wait that names the cause is the one that reports.
@@ -355,10 +357,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
         }
         for (int s = 0; s < kQueue; ++s) {
             mbar_init(q_full(s), 1);        // producer
-            mbar_init(q_empty(s), 11);      // MMA issuer, 8 epilogue warps, publisher, token-tile producer
+            mbar_init(q_empty(s), 12);      // weight producer, MMA issuer, 8 epilogue warps, publisher, token-tile producer
         }
         for (int s = 0; s < kMailSlots; ++s) mbar_init(mail_bar(s), 1);   // the pair leader's scheduler
         mbar_init(way_out_bar, 1);                                        // one commit, only after a wait gave up
+        mbar_init(claim_bar, 1);                                          // the weight producer, once per unit
         for (int s = 0; s < kMaxStagesA; ++s) {
             mbar_init(full_c(s), 2);    // the expect_tx arrivals of the weight producer and of the token-tile producer
             mbar_init(empty_c(s), 1);   // one tcgen05.commit
@@ -385,7 +388,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     // kernel holding some SMs) still cannot wait on a unit that nobody is working on.  The draw is
     // issued here and its answer used after the unit table is built, which hides the round trip.
     int first_draw = 0;
-    if (warp == 0 && lane == 0 && (!kPair || cluster_ctarank() == 0)) first_draw = atomicAdd(P.next_unit, 1);
+    if (warp == 6 && lane == 1 && (!kPair || cluster_ctarank() == 0)) first_draw = atomicAdd(P.next_unit, 1);
 
     // ---- unit table from the router's outputs -----------------------------------------------
     // Thread e reads expert e's class, count and offset (independent loads: one round trip to
@@ -560,54 +563,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
             uint32_t filled = 0;        // bit s: stage s has been filled at least once
             bool ok = true;
-            // Publishes unit number `j` of this CTA (or the end marker) to the other roles.
-            auto push_unit = [&](int j, const Unit& un) -> bool {
-                const int slot = j % kQueue;
-                if (!mbar_wait(q_empty(slot), ((j / kQueue) & 1) ^ 1, abort_flag, kWaitLimitNs)) {
-                    report_timeout(P.status, abort_flag, kSiteQueue);
-                    return false;
-                }
-                *reinterpret_cast<Unit*>(unit_queue + slot * 16) = un;
-                mbar_arrive(q_full(slot));          // release: the record is visible to whoever acquires
-                return true;
-            };
-            // In a CTA pair the
-            // leader draws from the counter and posts the index into the other CTA's mailbox (a
-            // remote store released by a remote mbarrier arrival).  The other CTA's loads gate the
-            // leader's MMAs, so it is never more than five draws behind and eight slots suffice.
-            int draws = 0;
-            auto draw = [&]() -> int {
-                if (draws == 0) return first_draw;      // drawn before the unit table was built
-                return atomicAdd(P.next_unit, 1);
-            };
-            auto take_next = [&]() -> int {
-                if (!kPair) {
-                    const int idx = draw();
-                    ++draws;
-                    return idx;
-                }
-                const int slot = draws % kMailSlots;
-                const uint32_t parity = (draws / kMailSlots) & 1;
-                if (rank == 0) {
-                    const int idx = draw();
-                    ++draws;
-                    st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(mail) + slot), 1), static_cast<uint32_t>(idx));
-                    mbar_arrive_cluster(map_to_cta(mail_bar(slot), 1));
-                    return idx;
-                }
-                ++draws;
-                if (!mbar_wait_cluster(mail_bar(slot), parity, abort_flag, kWaitLimitNs)) {
-                    report_timeout(P.status, abort_flag, kSiteQueue);
-                    return 0x7fffffff;
-                }
-                return mail[slot];
-            };
-            Unit cur, nxt;
-            const int u = take_next();
-            cur.id = -1;
-            if (u < ut.total_units) cur = ut.decode(u);
-            ok = push_unit(0, cur);
-            int u_ahead = cur.id >= 0 ? take_next() : 0;   // used a few K blocks later
+            Unit cur = pop_unit(0, false);
             for (int it = 0; ok && cur.id >= 0; ++it) {
                 const Unit un = cur;
                 trace_mark(P, it, 0, static_cast<unsigned long long>(un.id));
@@ -638,19 +594,14 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 const int w_row = un.e * N + un.n0 + (kPair ? static_cast<int>(rank) * kTileRows : 0);
                 const uint32_t tx_bytes = un.tiles * kABytes;
                 const bool trace_on = P.trace != nullptr;
-                bool next_ready = false;
+                bool next_asked = false;
                 for (int kb = kb0; kb < kb1; kb += kKps) {
-                    if (!next_ready && (kb1 - kb <= kClaimAhead || kb + kKps >= kb1)) {
-                        // take, decode and publish the next unit while this one's last loads are in flight
+                    if (!next_asked && (kb1 - kb <= kClaimAhead || kb + kKps >= kb1)) {
+                        // the scheduler may take the next unit now, while this one's last loads are in flight
                         // (not earlier: a unit claimed at the start of a long one would sit unworked for
                         // the whole of it while other SMs run out of units of its kind)
-                        nxt.id = -1;
-                        if (u_ahead < ut.total_units) {
-                            nxt = ut.decode(u_ahead);
-                            u_ahead = take_next();
-                        }
-                        if (!push_unit(it + 1, nxt)) { ok = false; break; }
-                        next_ready = true;
+                        mbar_arrive(claim_bar);
+                        next_asked = true;
                     }
                     if (!mbar_wait(empty0 + 8u * stage, ((fill_bits >> (stage + bit0)) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteProducerEmpty);
@@ -675,7 +626,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     if (++stage == na) stage = 0;
                 }
                 trace_time(P, it, 2);
-                cur = nxt;
+                if (ok) cur = pop_unit(it + 1, false);
             }
             // A CTA must not exit while bulk copies into its shared memory are outstanding.  After a
             // normal run every fill has been consumed (the MMA issuer waited for it) and these probes
@@ -1108,6 +1059,73 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     __threadfence();
                     atomicAdd(P.part_done + un.tile_idx, 1);
                 }
+            }
+        } else if (lane == 1) {
+            // ---- scheduler: draws units from the device-wide counter, decodes them and queues them for the
+            // other roles.  A thread of its own, because a draw is an atomic whose answer takes half a
+            // microsecond or more to come back while TMA loads fill the memory system, and decoding a unit is
+            // another half: on the weight producer's thread (where this used to run) that was a microsecond per
+            // unit in which no load was issued.  The producer says when it wants the next unit.
+            bool ok = true;
+            // Publishes unit number `j` of this CTA (or the end marker) to the other roles.
+            auto push_unit = [&](int j, const Unit& un) -> bool {
+                const int slot = j % kQueue;
+                if (!mbar_wait(q_empty(slot), ((j / kQueue) & 1) ^ 1, abort_flag, kWaitLimitNs)) {
+                    report_timeout(P.status, abort_flag, kSiteQueue);
+                    return false;
+                }
+                *reinterpret_cast<Unit*>(unit_queue + slot * 16) = un;
+                mbar_arrive(q_full(slot));          // release: the record is visible to whoever acquires
+                return true;
+            };
+            // In a CTA pair the
+            // leader draws from the counter and posts the index into the other CTA's mailbox (a
+            // remote store released by a remote mbarrier arrival).  The other CTA's loads gate the
+            // leader's MMAs, so it is never more than five draws behind and eight slots suffice.
+            int draws = 0;
+            auto draw = [&]() -> int {
+                if (draws == 0) return first_draw;      // drawn before the unit table was built
+                return atomicAdd(P.next_unit, 1);
+            };
+            auto take_next = [&]() -> int {
+                if (!kPair) {
+                    const int idx = draw();
+                    ++draws;
+                    return idx;
+                }
+                const int slot = draws % kMailSlots;
+                const uint32_t parity = (draws / kMailSlots) & 1;
+                if (rank == 0) {
+                    const int idx = draw();
+                    ++draws;
+                    st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(mail) + slot), 1), static_cast<uint32_t>(idx));
+                    mbar_arrive_cluster(map_to_cta(mail_bar(slot), 1));
+                    return idx;
+                }
+                ++draws;
+                if (!mbar_wait_cluster(mail_bar(slot), parity, abort_flag, kWaitLimitNs)) {
+                    report_timeout(P.status, abort_flag, kSiteQueue);
+                    return 0x7fffffff;
+                }
+                return mail[slot];
+            };
+            Unit nxt;
+            const int u = take_next();
+            nxt.id = -1;
+            if (u < ut.total_units) nxt = ut.decode(u);
+            ok = push_unit(0, nxt);
+            int u_ahead = nxt.id >= 0 ? take_next() : 0;   // its answer is used one unit later
+            for (int j = 1; ok && nxt.id >= 0; ++j) {
+                if (!mbar_wait(claim_bar, (j - 1) & 1, abort_flag, kWaitLimitNs)) {   // the producer is in unit j - 1
+                    report_timeout(P.status, abort_flag, kSiteQueue);
+                    break;
+                }
+                nxt.id = -1;
+                if (u_ahead < ut.total_units) {
+                    nxt = ut.decode(u_ahead);
+                    u_ahead = take_next();
+                }
+                ok = push_unit(j, nxt);
             }
         }
     }
