@@ -126,9 +126,7 @@ int monde_classify_top_h(const monde_problem* p, const int32_t* counts, double a
  * order); Section 4.1 (drop-less, padding-less routing: no capacity, no padded slot).
  *   pos(a) = offsets[e_a] + #{a' < a : e_a' = e_a};  perm[pos] = a;  inv_perm[a] = pos
  *   x_perm[pos,:] = x[a / top_k,:]
- * in : x [T,d_model]; topk_idx [T,k]; offsets [E+1]; and, inside `ws`, the per-chunk expert
- *      counts that monde_route left there: call it after monde_route for the same tokens, on the
- *      same workspace and stream
+ * in : x [T,d_model]; topk_idx [T,k]; offsets [E+1]
  * out: perm [A], inv_perm [A] int32; x_perm [A,d_model] (dtype)
  */
 int monde_permute(const monde_problem* p, const void* x, const int32_t* topk_idx,

@@ -31,16 +31,10 @@ struct WsLayout {
     size_t part_done_bytes;
     size_t partials_off;    // fp32 partial tiles of the K-split cold second-layer units
     size_t partials_bytes;
-    // Router scratch, written by monde_route and read by monde_permute (same workspace, same stream):
-    size_t chunk_counts_off;   // uint8 [n_chunks][E]: assignments of each 16-token chunk to each expert
-    size_t super_before_off;   // int32 [n_super][E]: assignments to each expert in all earlier super-chunks
     size_t logits_off;         // fp32 [T][kMaxExperts]: gate logits of small batches, between the two phases of the split router
     size_t stage_off;          // [T][top_k][d_model] in the problem dtype: expert outputs in token order (fused combine, top_k > 1)
-    int n_chunks, n_super;
     size_t total;
 };
-constexpr int kChunkTokens = 16;     // tokens per router CTA = one chunk of the permutation
-constexpr int kSuperChunks = 16;     // chunks per super-chunk
 constexpr int kSplitRouteMaxTokens = 256;   // batches up to this size take the split router (experts dealt over CTAs)
 // The header (first kHidden bytes) holds everything that must be zero between calls: the
 // status word, the CTA ticket (kCounters), one int32 per token tile that counts finished
@@ -79,12 +73,8 @@ inline WsLayout ws_layout(const monde_problem& p) {
     l.part_done_bytes = split > 1 ? (cold_tiles * 4 + 1023) / 1024 * 1024 : 0;
     l.partials_off = WsLayout::kHidden + l.hidden_bytes;
     l.partials_bytes = part;
-    l.n_chunks = (p.T + kChunkTokens - 1) / kChunkTokens;
-    l.n_super = (l.n_chunks + kSuperChunks - 1) / kSuperChunks;
     auto round256 = [](size_t v) { return (v + 255) / 256 * 256; };
-    l.chunk_counts_off = round256(l.partials_off + l.partials_bytes);
-    l.super_before_off = round256(l.chunk_counts_off + static_cast<size_t>(l.n_chunks) * p.E);
-    l.logits_off = round256(l.super_before_off + static_cast<size_t>(l.n_super) * p.E * 4);
+    l.logits_off = round256(l.partials_off + l.partials_bytes);
     const size_t logits_bytes = p.T <= kSplitRouteMaxTokens ? static_cast<size_t>(p.T) * kMaxExperts * 4 : 0;
     l.stage_off = round256(l.logits_off + logits_bytes);
     const size_t stage_bytes = (p.top_k > 1 && p.dtype == MONDE_BF16) ? A * p.d_model * elem_bytes(p.dtype) : 0;
@@ -155,7 +145,7 @@ int launch_route(const monde_problem& p, const void* x, const void* Wg, const fl
                  int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, void* ws, cudaStream_t s);
 int launch_classify_top_h(const monde_problem& p, double share, const int32_t* counts, uint8_t* cls,
                           int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, cudaStream_t s);
-// Reads the per-chunk expert counts that launch_route left in the same workspace.
+// Large batches use a dead part of the workspace (the hidden-activation region) for per-expert prefix counts.
 int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_idx, const int32_t* offsets,
                    int32_t* perm, int32_t* inv_perm, void* x_perm, const void* ws, cudaStream_t s);
 int launch_combine(const monde_problem& p, const void* y_perm, const int32_t* inv_perm,

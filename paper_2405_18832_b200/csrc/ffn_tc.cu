@@ -72,7 +72,7 @@ constexpr int kHotTokTile = 256;
 constexpr int kTilesPerUnit = 2;      // a unit covers two 128-feature tiles that share one token tile
 constexpr int kTileBytes = 192 * 1024;
 constexpr int kMailSlots = 8;        // unit indices in flight from the leader of a CTA pair to the other CTA
-constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue + kMailSlots + 1 + 2 * kMaxStagesA + 1;   // + the MMA issuer's way-out barrier + the shared barriers of lockstep rings
+constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue + kMailSlots + 1;   // + the MMA issuer's way-out barrier
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
 constexpr int kStageOutBytes = 2 * 2 * 16 * kTileRows * 2;   // per epilogue warp set: two staging buffers of 16 tokens x 128 features
 constexpr int kSmemBytes = 1024 + kTileBytes + kNumBars * 8 + 64 + kQueue * 64 + kTableInts * 4 + kStageOutBytes + 16;
@@ -318,12 +318,6 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     auto q_empty = [&](int s) { return bar0 + 8u * (kRingBars + 6 + kQueue + s); };
     auto mail_bar = [&](int s) { return bar0 + 8u * (kRingBars + 6 + 2 * kQueue + s); };
     const uint32_t way_out_bar = bar0 + 8u * (kRingBars + 6 + 2 * kQueue + kMailSlots);
-    // Lockstep rings (cold class): weight stage s and token stage s are filled, used and freed together,
-    // so one "full" barrier (both producers arrive on it) and one "empty" barrier (one commit) serve both.
-    auto full_c = [&](int s) { return bar0 + 8u * (kRingBars + 7 + 2 * kQueue + kMailSlots + s); };
-    auto empty_c = [&](int s) { return bar0 + 8u * (kRingBars + 7 + 2 * kQueue + kMailSlots + kMaxStagesA + s); };
-    // the weight producer tells the scheduler that the unit it is loading is nearly issued: time to take the next one
-    const uint32_t claim_bar = bar0 + 8u * (kRingBars + 7 + 2 * kQueue + kMailSlots + 2 * kMaxStagesA);
     // Waits on another unit's results (hidden rows, partial tiles) give up after wait_ns; waits on the
     // CTA's own barriers, which can only be waiting for one of those, after twice as long, so that the
     // wait that names the cause is the one that reports.
@@ -357,15 +351,10 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
         }
         for (int s = 0; s < kQueue; ++s) {
             mbar_init(q_full(s), 1);        // producer
-            mbar_init(q_empty(s), 12);      // weight producer, MMA issuer, 8 epilogue warps, publisher, token-tile producer
+            mbar_init(q_empty(s), 11);      // MMA issuer, 8 epilogue warps, publisher, token-tile producer
         }
         for (int s = 0; s < kMailSlots; ++s) mbar_init(mail_bar(s), 1);   // the pair leader's scheduler
         mbar_init(way_out_bar, 1);                                        // one commit, only after a wait gave up
-        mbar_init(claim_bar, 1);                                          // the weight producer, once per unit
-        for (int s = 0; s < kMaxStagesA; ++s) {
-            mbar_init(full_c(s), 2);    // the expect_tx arrivals of the weight producer and of the token-tile producer
-            mbar_init(empty_c(s), 1);   // one tcgen05.commit
-        }
         fence_barrier_init();
         for (int l = 0; l < 2; ++l) {
             prefetch_tensormap(&M.w[l][0]);
@@ -388,7 +377,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     // kernel holding some SMs) still cannot wait on a unit that nobody is working on.  The draw is
     // issued here and its answer used after the unit table is built, which hides the round trip.
     int first_draw = 0;
-    if (warp == 6 && lane == 1 && (!kPair || cluster_ctarank() == 0)) first_draw = atomicAdd(P.next_unit, 1);
+    if (warp == 0 && lane == 0 && (!kPair || cluster_ctarank() == 0)) first_draw = atomicAdd(P.next_unit, 1);
 
     // ---- unit table from the router's outputs -----------------------------------------------
     // Thread e reads expert e's class, count and offset (independent loads: one round trip to
@@ -489,30 +478,19 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     // token-tile stages fetched just in time, and all remaining shared memory as weight stages
     // in flight.  (With one combined ring the hot class had 48 KB of weights in flight per SM
     // and ran at the latency limit, 77 GB/s of fill per SM.)
-    // The cold class of single CTAs runs its two rings in lockstep (as many token stages as weight stages,
-    // shared barriers): its K blocks are short (N <= 64), so every barrier round trip and commit taken off
-    // the MMA-issuing thread counts.
-    struct Geom { int a_bytes, b_bytes, na, nb, b_base, lock; };
+    struct Geom { int a_bytes, b_bytes, na, nb, b_base; };
     auto geom_of = [&](int g) {
         Geom r;
         r.a_bytes = kPair ? kKps * kABytes : ut.tpu[g] * kABytes;                        // per CTA
         r.b_bytes = ((g & 2) ? P.cold_tile : kHotTokTile) * (kPair ? kKps * 64 : 128);   // a pair holds half the tokens each
-        r.lock = !kPair && (g & 2) != 0;
-        if (r.lock) {
-            r.na = r.nb = min(kMaxStagesA, kTileBytes / (r.a_bytes + r.b_bytes));
-        } else {
-            r.nb = (g & 2) ? 4 : 3;
-            r.na = min(kMaxStagesA, (kTileBytes - r.nb * r.b_bytes) / r.a_bytes);
-        }
+        r.nb = (g & 2) ? 4 : 3;
+        r.na = min(kMaxStagesA, (kTileBytes - r.nb * r.b_bytes) / r.a_bytes);
         r.b_base = r.na * r.a_bytes;
         return r;
     };
     auto same_geom = [](const Geom& x, const Geom& y) {
-        return x.a_bytes == y.a_bytes && x.b_bytes == y.b_bytes && x.na == y.na && x.nb == y.nb && x.lock == y.lock;
+        return x.a_bytes == y.a_bytes && x.b_bytes == y.b_bytes && x.na == y.na && x.nb == y.nb;
     };
-    // Bit index of a stage in the producers' and the issuer's parity masks: the shared barriers of the
-    // lockstep rings are counted apart from each ring's own.
-    constexpr int kLockBit = kMaxStagesA;
 
     // The producer decodes every unit once, one unit ahead of its loads, and hands the decoded
     // record to the other roles through a small shared-memory queue (decoding costs about half
@@ -563,7 +541,54 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             uint32_t fill_bits = 0;     // bit s: parity of the number of fills of stage s
             uint32_t filled = 0;        // bit s: stage s has been filled at least once
             bool ok = true;
-            Unit cur = pop_unit(0, false);
+            // Publishes unit number `j` of this CTA (or the end marker) to the other roles.
+            auto push_unit = [&](int j, const Unit& un) -> bool {
+                const int slot = j % kQueue;
+                if (!mbar_wait(q_empty(slot), ((j / kQueue) & 1) ^ 1, abort_flag, kWaitLimitNs)) {
+                    report_timeout(P.status, abort_flag, kSiteQueue);
+                    return false;
+                }
+                *reinterpret_cast<Unit*>(unit_queue + slot * 16) = un;
+                mbar_arrive(q_full(slot));          // release: the record is visible to whoever acquires
+                return true;
+            };
+            // In a CTA pair the
+            // leader draws from the counter and posts the index into the other CTA's mailbox (a
+            // remote store released by a remote mbarrier arrival).  The other CTA's loads gate the
+            // leader's MMAs, so it is never more than five draws behind and eight slots suffice.
+            int draws = 0;
+            auto draw = [&]() -> int {
+                if (draws == 0) return first_draw;      // drawn before the unit table was built
+                return atomicAdd(P.next_unit, 1);
+            };
+            auto take_next = [&]() -> int {
+                if (!kPair) {
+                    const int idx = draw();
+                    ++draws;
+                    return idx;
+                }
+                const int slot = draws % kMailSlots;
+                const uint32_t parity = (draws / kMailSlots) & 1;
+                if (rank == 0) {
+                    const int idx = draw();
+                    ++draws;
+                    st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(mail) + slot), 1), static_cast<uint32_t>(idx));
+                    mbar_arrive_cluster(map_to_cta(mail_bar(slot), 1));
+                    return idx;
+                }
+                ++draws;
+                if (!mbar_wait_cluster(mail_bar(slot), parity, abort_flag, kWaitLimitNs)) {
+                    report_timeout(P.status, abort_flag, kSiteQueue);
+                    return 0x7fffffff;
+                }
+                return mail[slot];
+            };
+            Unit cur, nxt;
+            const int u = take_next();
+            cur.id = -1;
+            if (u < ut.total_units) cur = ut.decode(u);
+            ok = push_unit(0, cur);
+            int u_ahead = cur.id >= 0 ? take_next() : 0;   // used a few K blocks later
             for (int it = 0; ok && cur.id >= 0; ++it) {
                 const Unit un = cur;
                 trace_mark(P, it, 0, static_cast<unsigned long long>(un.id));
@@ -571,14 +596,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     const Geom g2 = geom_of(un.cold * 2 + un.layer);
                     if (cls < 0 || !same_geom(g2, gm)) {
                         // geometry switch: every stage filled so far must have been consumed
-                        for (int s = 0; ok && cls >= 0 && s < gm.na; ++s) {
-                            const int bit = s + (gm.lock ? kLockBit : 0);
-                            if (!mbar_wait(gm.lock ? empty_c(s) : empty_a(s), ((fill_bits >> bit) & 1u) ^ 1u, abort_flag,
-                                           kWaitLimitNs)) {
+                        for (int s = 0; ok && cls >= 0 && s < gm.na; ++s)
+                            if (!mbar_wait(empty_a(s), ((fill_bits >> s) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                                 report_timeout(P.status, abort_flag, kSiteDrain);
                                 ok = false;
                             }
-                        }
                         if (!ok) break;
                         gm = g2;
                         stage = 0;
@@ -589,21 +611,24 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 const int N = un.layer ? P.d_model : P.d_ff;
                 // loop state in registers (see the MMA issuer)
                 const int kb0 = un.kb0, kb1 = un.kb1, a_bytes = gm.a_bytes, na = gm.na;
-                const int bit0 = gm.lock ? kLockBit : 0;
-                const uint32_t full0 = gm.lock ? full_c(0) : full_a(0), empty0 = gm.lock ? empty_c(0) : empty_a(0);
                 const int w_row = un.e * N + un.n0 + (kPair ? static_cast<int>(rank) * kTileRows : 0);
                 const uint32_t tx_bytes = un.tiles * kABytes;
                 const bool trace_on = P.trace != nullptr;
-                bool next_asked = false;
+                bool next_ready = false;
                 for (int kb = kb0; kb < kb1; kb += kKps) {
-                    if (!next_asked && (kb1 - kb <= kClaimAhead || kb + kKps >= kb1)) {
-                        // the scheduler may take the next unit now, while this one's last loads are in flight
+                    if (!next_ready && (kb1 - kb <= kClaimAhead || kb + kKps >= kb1)) {
+                        // take, decode and publish the next unit while this one's last loads are in flight
                         // (not earlier: a unit claimed at the start of a long one would sit unworked for
                         // the whole of it while other SMs run out of units of its kind)
-                        mbar_arrive(claim_bar);
-                        next_asked = true;
+                        nxt.id = -1;
+                        if (u_ahead < ut.total_units) {
+                            nxt = ut.decode(u_ahead);
+                            u_ahead = take_next();
+                        }
+                        if (!push_unit(it + 1, nxt)) { ok = false; break; }
+                        next_ready = true;
                     }
-                    if (!mbar_wait(empty0 + 8u * stage, ((fill_bits >> (stage + bit0)) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
+                    if (!mbar_wait(empty_a(stage), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteProducerEmpty);
                         ok = false;
                         break;
@@ -617,16 +642,16 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         for (int j = 0; j < nk; ++j)
                             tma_load_2d_pair(a_dst + j * kABytes, mw, bar0_leader + 8u * stage, (kb + j) * kBlockK, w_row, pol_w);
                     } else {
-                        const uint32_t full = full0 + 8u * stage;
+                        const uint32_t full = full_a(stage);
                         mbar_arrive_expect_tx(full, tx_bytes);
                         tma_load_2d(a_dst, mw, full, kb * kBlockK, w_row, pol_w);
                     }
-                    fill_bits ^= 1u << (stage + bit0);
-                    filled |= 1u << (stage + bit0);
+                    fill_bits ^= 1u << stage;
+                    filled |= 1u << stage;
                     if (++stage == na) stage = 0;
                 }
                 trace_time(P, it, 2);
-                if (ok) cur = pop_unit(it + 1, false);
+                cur = nxt;
             }
             // A CTA must not exit while bulk copies into its shared memory are outstanding.  After a
             // normal run every fill has been consumed (the MMA issuer waited for it) and these probes
@@ -634,11 +659,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
             // them, bounded by time alone.  (Pairs: the leader's barriers count both CTAs' copies and
             // the cluster barrier in the teardown holds the other CTA until the leader is through.)
             if (!kPair || rank == 0)
-                for (int s = 0; s < kMaxStagesA; ++s) {
+                for (int s = 0; s < kMaxStagesA; ++s)
                     if ((filled >> s) & 1u) mbar_wait_deadline(full_a(s), ((fill_bits >> s) & 1u) ^ 1u, kDrainLimitNs);
-                    if ((filled >> (s + kLockBit)) & 1u)
-                        mbar_wait_deadline(full_c(s), ((fill_bits >> (s + kLockBit)) & 1u) ^ 1u, kDrainLimitNs);
-                }
         }
     } else if (warp == 7) {
         // ---- token-tile producer (operand B: rows of x_perm or of the hidden activations) -------
@@ -654,14 +676,11 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 if (un.cold * 2 + un.layer != cls) {
                     const Geom g2 = geom_of(un.cold * 2 + un.layer);
                     if (cls < 0 || !same_geom(g2, gm)) {
-                        for (int s = 0; ok && cls >= 0 && s < gm.nb; ++s) {
-                            const int bit = s + (gm.lock ? kLockBit : 0);
-                            if (!mbar_wait(gm.lock ? empty_c(s) : empty_b(s), ((fill_bits >> bit) & 1u) ^ 1u, abort_flag,
-                                           kWaitLimitNs)) {
+                        for (int s = 0; ok && cls >= 0 && s < gm.nb; ++s)
+                            if (!mbar_wait(empty_b(s), ((fill_bits >> s) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                                 report_timeout(P.status, abort_flag, kSiteDrain);
                                 ok = false;
                             }
-                        }
                         if (!ok) break;
                         gm = g2;
                         stage = 0;
@@ -689,10 +708,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 // loop state in registers (see the MMA issuer)
                 const int kb0 = un.kb0, kb1 = un.kb1, nt = un.nt, row0 = un.row0, b_bytes = gm.b_bytes, nb = gm.nb;
                 const uint32_t b_ring = tiles_u32 + gm.b_base;
-                const int bit0 = gm.lock ? kLockBit : 0;
-                const uint32_t full0 = gm.lock ? full_c(0) : full_b(0), empty0 = gm.lock ? empty_c(0) : empty_b(0);
                 for (int kb = kb0; kb < kb1; kb += kKps) {
-                    if (!mbar_wait(empty0 + 8u * stage, ((fill_bits >> (stage + bit0)) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
+                    if (!mbar_wait(empty_b(stage), ((fill_bits >> stage) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         report_timeout(P.status, abort_flag, kSiteProducerEmpty);
                         ok = false;
                         break;
@@ -713,7 +730,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                             for (; half - j >= 8; j += 8) tma_load_2d_pair(dst + j * 128, mi, full, x, r0 + j, pol_x);
                         }
                     } else {
-                        const uint32_t full = full0 + 8u * stage;
+                        const uint32_t full = full_b(stage);
                         mbar_arrive_expect_tx(full, nt * 128);
                         int j = 0;
                         for (; nt - j >= 256; j += 256)
@@ -723,19 +740,15 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         for (; nt - j >= 16; j += 16)
                             tma_load_2d(b_dst + j * 128, mi, full, kb * kBlockK, row0 + j, pol_x);
                     }
-                    fill_bits ^= 1u << (stage + bit0);
-                    filled |= 1u << (stage + bit0);
+                    fill_bits ^= 1u << stage;
+                    filled |= 1u << stage;
                     if (++stage == nb) stage = 0;
                 }
             }
             // copies in flight into this CTA's shared memory must land before it exits (see the weight producer)
-            if (!kPair || rank == 0) {
+            if (!kPair || rank == 0)
                 for (int s = 0; s < kMaxStagesB; ++s)
                     if ((filled >> s) & 1u) mbar_wait_deadline(full_b(s), ((fill_bits >> s) & 1u) ^ 1u, kDrainLimitNs);
-                for (int s = 0; s < kMaxStagesA; ++s)
-                    if ((filled >> (s + kLockBit)) & 1u)
-                        mbar_wait_deadline(full_c(s), ((fill_bits >> (s + kLockBit)) & 1u) ^ 1u, kDrainLimitNs);
-            }
         }
     } else if (warp == 1) {
         // ---- MMA issuer --------------------------------------------------------------
@@ -778,14 +791,12 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 const uint32_t acc1 = tmem_base + (kPair ? b * 256 : acc_col(un, b, 1));
                 const bool trace_on = P.trace != nullptr;
                 bool stage_ready = false;       // the next K block's barriers were probed during this one's MMAs
-                const bool lock = gm.lock != 0;  // lockstep rings: sa == sb, one barrier pair per stage, parities in use_a
                 unsigned long long waited = 0;   // diagnostic timeline: time spent waiting for operands
                 for (int kb = kb0; kb < kb1; kb += kKps) {
                     const unsigned long long w0 = trace_on && !stage_ready ? global_timer_ns() : 0;
                     if (!stage_ready &&
-                        (lock ? !mbar_wait(full_c(sa), (use_a >> (sa + kLockBit)) & 1u, abort_flag, kWaitLimitNs)
-                              : (!mbar_wait(full_a(sa), (use_a >> sa) & 1u, abort_flag, kWaitLimitNs) ||
-                                 !mbar_wait(full_b(sb), (use_b >> sb) & 1u, abort_flag, kWaitLimitNs)))) {
+                        (!mbar_wait(full_a(sa), (use_a >> sa) & 1u, abort_flag, kWaitLimitNs) ||
+                         !mbar_wait(full_b(sb), (use_b >> sb) & 1u, abort_flag, kWaitLimitNs))) {
                         report_timeout(P.status, abort_flag, kSiteMmaFull);
                         ok = false;
                         break;
@@ -815,30 +826,17 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         // rings have at least three stages, so the next stage is not this one and its use
                         // bit is still that of its next fill; past the unit's last K block the answer is unused
                         const int sa_next = sa + 1 == na ? 0 : sa + 1, sb_next = sb + 1 == nb ? 0 : sb + 1;
-                        // probes of the next stage, this block's MMAs (the second feature tile shares the token
-                        // tile), the commits that free the stage(s): one instruction sequence, answers read last
-                        bool next_full;
-                        if (lock) {
-                            const uint32_t pb = full_c(sa_next), pp = (use_a >> (sa_next + kLockBit)) & 1u, cb = empty_c(sa);
-                            next_full = tiles == 2
-                                ? umma_bf16_kblock<2, 1>(acc0, acc1, a_desc, b_desc, idesc, later, pb, pp, 0, 0, cb, 0)
-                                : umma_bf16_kblock<1, 1>(acc0, acc1, a_desc, b_desc, idesc, later, pb, pp, 0, 0, cb, 0);
-                            use_a ^= 1u << (sa + kLockBit);
-                        } else {
-                            const uint32_t pa = full_a(sa_next), ppa = (use_a >> sa_next) & 1u;
-                            const uint32_t pb = full_b(sb_next), ppb = (use_b >> sb_next) & 1u;
-                            next_full = tiles == 2
-                                ? umma_bf16_kblock<2, 2>(acc0, acc1, a_desc, b_desc, idesc, later, pa, ppa, pb, ppb,
-                                                         empty_a(sa), empty_b(sb))
-                                : umma_bf16_kblock<1, 2>(acc0, acc1, a_desc, b_desc, idesc, later, pa, ppa, pb, ppb,
-                                                         empty_a(sa), empty_b(sb));
-                            use_a ^= 1u << sa;
-                            use_b ^= 1u << sb;
+                        stage_ready = umma_bf16_x4_probe(acc0, a_desc, b_desc, idesc, later, full_a(sa_next),
+                                                         (use_a >> sa_next) & 1u, full_b(sb_next), (use_b >> sb_next) & 1u) &&
+                                      kb + 1 < kb1;
+                        if (tiles == 2) {                  // the second feature tile shares the token tile
+                            const uint64_t a1_desc = smem_desc_sw128(a_addr + kABytes);
+#pragma unroll
+                            for (int k4 = 0; k4 < kBlockK / 16; ++k4)
+                                umma_bf16(acc1, a1_desc + 2 * k4, b_desc + 2 * k4, idesc, later | (k4 != 0));
                         }
-                        stage_ready = next_full && kb + 1 < kb1;
-                        if (++sa == na) sa = 0;
-                        if (++sb == nb) sb = 0;
-                        continue;
+                        umma_commit(empty_a(sa));   // both stages reusable once these MMAs finish
+                        umma_commit(empty_b(sb));
                     }
                     use_a ^= 1u << sa;
                     use_b ^= 1u << sb;
@@ -1059,73 +1057,6 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                     __threadfence();
                     atomicAdd(P.part_done + un.tile_idx, 1);
                 }
-            }
-        } else if (lane == 1) {
-            // ---- scheduler: draws units from the device-wide counter, decodes them and queues them for the
-            // other roles.  A thread of its own, because a draw is an atomic whose answer takes half a
-            // microsecond or more to come back while TMA loads fill the memory system, and decoding a unit is
-            // another half: on the weight producer's thread (where this used to run) that was a microsecond per
-            // unit in which no load was issued.  The producer says when it wants the next unit.
-            bool ok = true;
-            // Publishes unit number `j` of this CTA (or the end marker) to the other roles.
-            auto push_unit = [&](int j, const Unit& un) -> bool {
-                const int slot = j % kQueue;
-                if (!mbar_wait(q_empty(slot), ((j / kQueue) & 1) ^ 1, abort_flag, kWaitLimitNs)) {
-                    report_timeout(P.status, abort_flag, kSiteQueue);
-                    return false;
-                }
-                *reinterpret_cast<Unit*>(unit_queue + slot * 16) = un;
-                mbar_arrive(q_full(slot));          // release: the record is visible to whoever acquires
-                return true;
-            };
-            // In a CTA pair the
-            // leader draws from the counter and posts the index into the other CTA's mailbox (a
-            // remote store released by a remote mbarrier arrival).  The other CTA's loads gate the
-            // leader's MMAs, so it is never more than five draws behind and eight slots suffice.
-            int draws = 0;
-            auto draw = [&]() -> int {
-                if (draws == 0) return first_draw;      // drawn before the unit table was built
-                return atomicAdd(P.next_unit, 1);
-            };
-            auto take_next = [&]() -> int {
-                if (!kPair) {
-                    const int idx = draw();
-                    ++draws;
-                    return idx;
-                }
-                const int slot = draws % kMailSlots;
-                const uint32_t parity = (draws / kMailSlots) & 1;
-                if (rank == 0) {
-                    const int idx = draw();
-                    ++draws;
-                    st_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(mail) + slot), 1), static_cast<uint32_t>(idx));
-                    mbar_arrive_cluster(map_to_cta(mail_bar(slot), 1));
-                    return idx;
-                }
-                ++draws;
-                if (!mbar_wait_cluster(mail_bar(slot), parity, abort_flag, kWaitLimitNs)) {
-                    report_timeout(P.status, abort_flag, kSiteQueue);
-                    return 0x7fffffff;
-                }
-                return mail[slot];
-            };
-            Unit nxt;
-            const int u = take_next();
-            nxt.id = -1;
-            if (u < ut.total_units) nxt = ut.decode(u);
-            ok = push_unit(0, nxt);
-            int u_ahead = nxt.id >= 0 ? take_next() : 0;   // its answer is used one unit later
-            for (int j = 1; ok && nxt.id >= 0; ++j) {
-                if (!mbar_wait(claim_bar, (j - 1) & 1, abort_flag, kWaitLimitNs)) {   // the producer is in unit j - 1
-                    report_timeout(P.status, abort_flag, kSiteQueue);
-                    break;
-                }
-                nxt.id = -1;
-                if (u_ahead < ut.total_units) {
-                    nxt = ut.decode(u_ahead);
-                    u_ahead = take_next();
-                }
-                ok = push_unit(j, nxt);
             }
         }
     }

@@ -1,6 +1,6 @@
 // Stable counting-sort permutation of assignments into expert-contiguous order, fused
 // with the row gather.  Deterministic: positions follow from counts alone, never from
-// the order in which threads run.  The counts per 16-token chunk come from the router.
+// the order in which threads run.
 // Paper: Section 2.1 (routing to experts); Section 4.1 (drop-less, padding-less).
 #include "common.cuh"
 
@@ -8,34 +8,64 @@ namespace monde {
 
 namespace {
 
-constexpr int kThreads = 128;        // four warps
-constexpr int kRowsPerWarp = 4;      // rows a warp copies together
-constexpr int kMaxChunkRows = kChunkTokens * kMaxTopK;   // assignments of one chunk
+constexpr int kChunk = 16;           // assignments per CTA, ranked by half a warp
+constexpr int kThreads = 128;        // four warps, four rows each
+constexpr int kRowsPerWarp = kChunk / (kThreads / 32);
 
-// CTA c owns the assignments of chunk c (16 tokens, 16 * k assignments), the same chunks the router
-// CTAs own.  The position of assignment a with expert e is
-//     offsets[e] + (assignments to e in earlier super-chunks)           <- super_before, from the router's tail
-//                + (assignments to e in earlier chunks of this super-chunk)   <- at most 15 one-byte counts
-//                + (earlier assignments to e inside this chunk)         <- compared in shared memory
-// every term an integer read or counted in a fixed way: positions never depend on the order in which
-// threads or CTAs run, and no CTA looks at another chunk's assignment list.
+// CTA c owns assignments [c*kChunk, (c+1)*kChunk).  The number of earlier assignments to
+// each expert is recounted from topk_idx (at most A integers, L2-resident), which keeps
+// the kernel single-pass and free of inter-CTA ordering.  Small chunks give many CTAs and
+// every warp keeps the loads of its four rows in flight together, which is what matters
+// for a decode-sized batch where the whole gather is a few dozen rows.
+// Large batches: the recount of earlier assignments would grow quadratically, so it is cut at
+// super-chunk boundaries.  `super_before` [n_super][E] holds, per expert, the number of assignments in
+// all earlier super-chunks (two small kernels below build it); a CTA then recounts only from the start
+// of its own super-chunk.  Null for small batches: recount from assignment 0.
+constexpr int kSuper = 2048;         // assignments per super-chunk
+constexpr int kTwoLevelFrom = 8192;  // batches with more assignments take the two-level path
+
+__global__ void __launch_bounds__(256) super_histogram_kernel(int A, int E, const int32_t* __restrict__ topk_idx,
+                                                              int32_t* __restrict__ super_before) {
+    __shared__ int hist[kMaxExperts];
+    pdl_launch_dependents();
+    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) hist[e] = 0;
+    __syncthreads();
+    pdl_wait();
+    const int first = blockIdx.x * kSuper;
+    for (int a = first + threadIdx.x; a < min(A, first + kSuper); a += blockDim.x) atomicAdd(&hist[topk_idx[a]], 1);
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) super_before[static_cast<size_t>(blockIdx.x) * E + e] = hist[e];
+}
+
+// In place: counts per super-chunk -> exclusive prefix over super-chunks, one thread per expert.
+__global__ void __launch_bounds__(256) super_scan_kernel(int n_super, int E, int32_t* __restrict__ super_before) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int e = threadIdx.x;
+    if (e >= E) return;
+    int running = 0;
+    for (int s = 0; s < n_super; ++s) {
+        const int c = super_before[static_cast<size_t>(s) * E + e];
+        super_before[static_cast<size_t>(s) * E + e] = running;
+        running += c;
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
         int A, int E, int k, int d, const T* __restrict__ x, const int32_t* __restrict__ topk_idx,
-        const int32_t* __restrict__ offsets, const uint8_t* __restrict__ chunk_counts,
-        const int32_t* __restrict__ super_before, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
-        T* __restrict__ x_perm) {
-    __shared__ int s_e[kMaxChunkRows];
-    __shared__ int s_pos[kMaxChunkRows];
+        const int32_t* __restrict__ offsets, const int32_t* __restrict__ super_before,
+        int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, T* __restrict__ x_perm) {
+    __shared__ int before[kMaxExperts];   // assignments to e in earlier chunks
+    __shared__ int row_pos[kChunk];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int chunk = blockIdx.x;
-    const int rows_per_chunk = kChunkTokens * k;
-    const int first = chunk * rows_per_chunk;
-    const int n_rows = min(rows_per_chunk, A - first);
+    const int first = blockIdx.x * kChunk;
     pdl_launch_dependents();
+    for (int e = tid; e < kMaxExperts; e += kThreads) before[e] = 0;
+    __syncthreads();
     pdl_wait();
-    // The rows this warp will copy are known before their positions are: the first vectors of its first
-    // rows are requested now, so that trip to memory overlaps the position computation.
+    // The rows this warp will copy are known before their positions are: their first vectors are
+    // requested now, so that trip to memory overlaps the recount and the rank computation.
     constexpr int V = Vec16<T>::N;
     constexpr int kIter = 3;                         // vectors per lane and row in flight
     const int vec_per_row = d / V;
@@ -43,62 +73,78 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
     uint4 v[kIter][kRowsPerWarp];
 #pragma unroll
     for (int r = 0; r < kRowsPerWarp; ++r) {
-        const int a = warp * kRowsPerWarp + r;       // row of the chunk
-        src[r] = a < n_rows ? reinterpret_cast<const uint4*>(x + static_cast<int64_t>((first + a) / k) * d) : nullptr;
+        const int a = first + warp * kRowsPerWarp + r;
+        src[r] = a < A ? reinterpret_cast<const uint4*>(x + static_cast<int64_t>(a / k) * d) : nullptr;
     }
 #pragma unroll
     for (int it = 0; it < kIter; ++it)
 #pragma unroll
         for (int r = 0; r < kRowsPerWarp; ++r)
             if (src[r] != nullptr && lane + 32 * it < vec_per_row) v[it][r] = src[r][lane + 32 * it];
-    // positions: thread a handles assignment first + a
-    int e = -1, base = 0;
-    if (tid < n_rows) {
-        e = topk_idx[first + tid];
-        const int sc = chunk / kSuperChunks, c0 = sc * kSuperChunks;
-        base = offsets[e] + super_before[static_cast<size_t>(sc) * E + e];
-        int earlier = 0;
-#pragma unroll
-        for (int c = 0; c < kSuperChunks - 1; ++c)    // independent one-byte loads: one trip to L2
-            earlier += c0 + c < chunk ? static_cast<int>(__ldg(chunk_counts + static_cast<size_t>(c0 + c) * E + e)) : 0;
-        base += earlier;
-    }
-    if (tid < kMaxChunkRows) s_e[tid] = e;
+    const int recount_from = super_before != nullptr ? (first / kSuper) * kSuper : 0;
+    if (super_before != nullptr)
+        for (int e = tid; e < E; e += kThreads) before[e] = super_before[static_cast<size_t>(first / kSuper) * E + e];
     __syncthreads();
-    if (tid < n_rows) {
-        int rank = 0;
-        for (int a = 0; a < tid; ++a) rank += s_e[a] == e;
-        const int pos = base + rank;
-        perm[pos] = first + tid;
-        inv_perm[first + tid] = pos;
-        s_pos[tid] = pos;
-    }
-    __syncthreads();
-    // Row gather with 16-byte accesses; a warp's rows advance together, kIter vectors per lane and
-    // row requested before any is stored (one trip to memory per batch, not per vector).
-    for (int r0 = warp * kRowsPerWarp; r0 < n_rows; r0 += (kThreads / 32) * kRowsPerWarp) {
-        uint4* dst[kRowsPerWarp];
+    // Recount: the loads are batched (four 16-byte loads per thread in flight, 2048 assignments per
+    // trip to L2) because the last chunks look back over thousands of assignments and a load per
+    // loop iteration made them the critical path of the whole call.
+    if ((reinterpret_cast<uintptr_t>(topk_idx) & 15) == 0) {
+        const int4* src4 = reinterpret_cast<const int4*>(topk_idx + recount_from);   // both multiples of 16
+        const int n4 = (first - recount_from) >> 2;
+        for (int i = tid; i < n4; i += 4 * kThreads) {
+            int4 v[4];
 #pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r) {
-            const int a = r0 + r;
-            dst[r] = a < n_rows ? reinterpret_cast<uint4*>(x_perm + static_cast<int64_t>(s_pos[a]) * d) : nullptr;
-            if (r0 != warp * kRowsPerWarp)           // later row groups (k > 1): their sources were not set up above
-                src[r] = a < n_rows ? reinterpret_cast<const uint4*>(x + static_cast<int64_t>((first + a) / k) * d) : nullptr;
-        }
-        for (int i0 = lane; i0 < vec_per_row; i0 += 32 * kIter) {
-            if (i0 != lane || r0 != warp * kRowsPerWarp) {      // the very first batch is already in registers
-#pragma unroll
-                for (int it = 0; it < kIter; ++it)
-#pragma unroll
-                    for (int r = 0; r < kRowsPerWarp; ++r)
-                        if (dst[r] != nullptr && i0 + 32 * it < vec_per_row) v[it][r] = src[r][i0 + 32 * it];
+            for (int j = 0; j < 4; ++j) {
+                const int q = i + j * kThreads;
+                v[j] = q < n4 ? __ldg(src4 + q) : make_int4(-1, -1, -1, -1);
             }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (v[j].x < 0) continue;
+                atomicAdd(&before[v[j].x], 1);
+                atomicAdd(&before[v[j].y], 1);
+                atomicAdd(&before[v[j].z], 1);
+                atomicAdd(&before[v[j].w], 1);
+            }
+        }
+    } else {
+        for (int a = recount_from + tid; a < first; a += kThreads) atomicAdd(&before[topk_idx[a]], 1);
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const int a = first + lane;
+        const int e = (lane < kChunk && a < A) ? topk_idx[a] : -1;
+        const unsigned same = __match_any_sync(0xffffffffu, e);
+        int pos = -1;
+        if (e >= 0) {
+            pos = offsets[e] + before[e] + __popc(same & ((1u << lane) - 1u));
+            perm[pos] = a;
+            inv_perm[a] = pos;
+        }
+        if (lane < kChunk) row_pos[lane] = pos;
+    }
+    __syncthreads();
+    // Row gather with 16-byte accesses; the warp's rows advance together, kIter vectors per lane and
+    // row requested before any is stored (one trip to memory per batch, not per vector).
+    uint4* dst[kRowsPerWarp];
+#pragma unroll
+    for (int r = 0; r < kRowsPerWarp; ++r) {
+        const int p = row_pos[warp * kRowsPerWarp + r];
+        dst[r] = p >= 0 ? reinterpret_cast<uint4*>(x_perm + static_cast<int64_t>(p) * d) : nullptr;
+    }
+    for (int i0 = lane; i0 < vec_per_row; i0 += 32 * kIter) {
+        if (i0 != lane) {      // the first batch is already in registers
 #pragma unroll
             for (int it = 0; it < kIter; ++it)
 #pragma unroll
                 for (int r = 0; r < kRowsPerWarp; ++r)
-                    if (dst[r] != nullptr && i0 + 32 * it < vec_per_row) dst[r][i0 + 32 * it] = v[it][r];
+                    if (dst[r] != nullptr && i0 + 32 * it < vec_per_row) v[it][r] = src[r][i0 + 32 * it];
         }
+#pragma unroll
+        for (int it = 0; it < kIter; ++it)
+#pragma unroll
+            for (int r = 0; r < kRowsPerWarp; ++r)
+                if (dst[r] != nullptr && i0 + 32 * it < vec_per_row) dst[r][i0 + 32 * it] = v[it][r];
     }
 }
 
@@ -133,19 +179,27 @@ __global__ void __launch_bounds__(256) combine_kernel(
 
 int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_idx, const int32_t* offsets,
                    int32_t* perm, int32_t* inv_perm, void* x_perm, const void* ws, cudaStream_t s) {
+    // scratch for the two-level recount: ceil(A / 2048) * E int32 in the hidden-activation region, which is dead
+    // during this call (the expert FFN rewrites it before reading it)
+    int32_t* scratch = reinterpret_cast<int32_t*>(static_cast<char*>(const_cast<void*>(ws)) + WsLayout::kHidden);
     const int A = p.T * p.top_k;
-    const WsLayout L = ws_layout(p);
-    const char* base = static_cast<const char*>(ws);
-    const uint8_t* chunk_counts = reinterpret_cast<const uint8_t*>(base + L.chunk_counts_off);
-    const int32_t* super_before = reinterpret_cast<const int32_t*>(base + L.super_before_off);
+    const int grid = (A + kChunk - 1) / kChunk;
+    int32_t* super_before = nullptr;
+    if (A > kTwoLevelFrom) {
+        const int n_super = (A + kSuper - 1) / kSuper;
+        super_before = scratch;      // n_super * E int32
+        launch_pdl(super_histogram_kernel, dim3(n_super), dim3(256), 0, s, A, p.E, topk_idx, super_before);
+        launch_pdl(super_scan_kernel, dim3(1), dim3(256), 0, s, n_super, p.E, super_before);
+        count_launches(2);
+    }
     if (p.dtype == MONDE_BF16)
-        launch_pdl(permute_gather_kernel<__nv_bfloat16>, dim3(L.n_chunks), dim3(kThreads), 0, s,
-            A, p.E, p.top_k, p.d_model, static_cast<const __nv_bfloat16*>(x), topk_idx, offsets, chunk_counts,
-            super_before, perm, inv_perm, static_cast<__nv_bfloat16*>(x_perm));
+        launch_pdl(permute_gather_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), 0, s,
+            A, p.E, p.top_k, p.d_model, static_cast<const __nv_bfloat16*>(x), topk_idx, offsets, super_before, perm,
+            inv_perm, static_cast<__nv_bfloat16*>(x_perm));
     else
-        launch_pdl(permute_gather_kernel<float>, dim3(L.n_chunks), dim3(kThreads), 0, s,
-            A, p.E, p.top_k, p.d_model, static_cast<const float*>(x), topk_idx, offsets, chunk_counts, super_before,
-            perm, inv_perm, static_cast<float*>(x_perm));
+        launch_pdl(permute_gather_kernel<float>, dim3(grid), dim3(kThreads), 0, s,
+            A, p.E, p.top_k, p.d_model, static_cast<const float*>(x), topk_idx, offsets, super_before, perm, inv_perm,
+            static_cast<float*>(x_perm));
     return launched();
 }
 

@@ -2,15 +2,6 @@
 // shared-memory histogram / hot-cold classification / scan over experts.
 // Paper: Section 2.1 (gating network, score map, top-k routing); Section 2.2 (hot and
 // cold experts by token count); Eq. 5 (activated = at least one token).
-//
-// Every router CTA owns one chunk of 16 tokens.  It leaves the chunk's per-expert assignment
-// counts in the workspace (one byte each); the CTA that finishes last adds them up over
-// super-chunks of 16 chunks, which gives the per-expert totals (the histogram) and, for the
-// permutation that follows, the number of assignments to each expert in all earlier
-// super-chunks.  No CTA ever walks the assignment list again.
-// Batches of up to 256 tokens have too few chunks to occupy the GPU: their gate GEMM is dealt
-// over (chunk, 8 experts) CTAs that exchange logits through the workspace, and the CTA that
-// completes a chunk's logits does its softmax and top-k.
 #include "common.cuh"
 
 namespace monde {
@@ -32,11 +23,9 @@ __device__ __forceinline__ float warp_max(float v) {
 
 // Softmax over all E logits and the k best of them, for one token held by one warp.
 // logit[s] of lane l is expert s*32+l (-inf beyond E).
-// `chunk_hist` (shared memory, zeroed, one int per expert) counts the picks of the CTA's 16 tokens.
 __device__ __forceinline__ void softmax_topk_store(const float (&logit)[kSlots], int E, int k, int renorm,
                                                    int64_t t, int lane, int32_t* __restrict__ topk_idx,
-                                                   float* __restrict__ topk_w, float* __restrict__ probs,
-                                                   int* chunk_hist) {
+                                                   float* __restrict__ topk_w, float* __restrict__ probs) {
     float m = -INFINITY;
 #pragma unroll
     for (int s = 0; s < kSlots; ++s) m = fmaxf(m, logit[s]);
@@ -92,29 +81,51 @@ __device__ __forceinline__ void softmax_topk_store(const float (&logit)[kSlots],
             if (j < k) {
                 topk_idx[t * k + j] = sel_e[j];
                 topk_w[t * k + j] = renorm ? sel_p[j] / mass : sel_p[j];
-                atomicAdd(&chunk_hist[sel_e[j]], 1);      // integer count in shared memory: order-free
             }
         }
     }
 }
 
 struct HistArgs {
-    int T, E, theta;
-    int n_chunks, n_super;
+    int A, E, theta;
     int32_t* counts;
     int32_t* offsets;
     uint8_t* cls;
     int32_t* hot_ids;
     int32_t* cold_ids;
     int32_t* n_hot_cold;
-    int32_t* ticket;          // chunks whose routing is finished (left at zero)
-    uint8_t* chunk_counts;    // [n_chunks][E]
-    int32_t* super_before;    // [n_super][E]
+    int32_t* ticket;      // CTAs of the router that have finished (left at zero)
 };
 
-// Classification, compaction and exclusive scan over the per-expert totals in hist[] (shared
-// memory); run by the first warp of one CTA.
-__device__ void classify_scan(const HistArgs& h, const int* hist) {
+// Histogram of assignments per expert (shared-memory atomics on integers: the sum does
+// not depend on order), then classification, compaction and exclusive scan by one warp.
+// Runs in one CTA of any size.
+__device__ void histogram_classify_scan(const HistArgs& h, const int32_t* __restrict__ topk_idx, int* hist) {
+    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) hist[e] = 0;
+    __syncthreads();
+    // The loads are batched (four 16-byte loads per thread in flight): this runs in the last CTA
+    // alone, after everything else, and one load per loop iteration would put A / blockDim.x trips
+    // to L2 on the critical path of the call.
+    const int A4 = (reinterpret_cast<uintptr_t>(topk_idx) & 15) == 0 ? h.A >> 2 : 0;
+    const int4* idx4 = reinterpret_cast<const int4*>(topk_idx);
+    for (int i = threadIdx.x; i < A4; i += 4 * blockDim.x) {
+        int4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int q = i + j * blockDim.x;
+            v[j] = q < A4 ? __ldcg(idx4 + q) : make_int4(-1, -1, -1, -1);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (v[j].x < 0) continue;
+            atomicAdd(&hist[v[j].x], 1);
+            atomicAdd(&hist[v[j].y], 1);
+            atomicAdd(&hist[v[j].z], 1);
+            atomicAdd(&hist[v[j].w], 1);
+        }
+    }
+    for (int a = A4 * 4 + threadIdx.x; a < h.A; a += blockDim.x) atomicAdd(&hist[__ldcg(topk_idx + a)], 1);
+    __syncthreads();
     if (threadIdx.x >= 32) return;
     const int lane = threadIdx.x;
     // lane owns experts [lane*8, lane*8+8)
@@ -158,82 +169,40 @@ __device__ void classify_scan(const HistArgs& h, const int* hist) {
     }
 }
 
-// The tail of the routing call, run by one CTA after every chunk's counts are in the workspace:
-// per super-chunk sums of the chunk counts, their exclusive scan over super-chunks (what the
-// permutation needs) and the totals (the histogram), then classification and scan.  Integer sums
-// in a fixed order: nothing depends on which CTA runs this or when.
-__device__ void histogram_classify_scan(const HistArgs& h, int* hist) {
-    const int E = h.E;
-    // 1. super_before[sc][e] <- assignments of super-chunk sc to expert e (16 byte-sized loads in flight per thread)
-    for (int i = threadIdx.x; i < h.n_super * E; i += blockDim.x) {
-        const int sc = i / E, e = i - sc * E;
-        const int c0 = sc * kSuperChunks;
-        int sum = 0;
-#pragma unroll
-        for (int c = 0; c < kSuperChunks; ++c)
-            sum += c0 + c < h.n_chunks ? static_cast<int>(__ldcg(h.chunk_counts + static_cast<size_t>(c0 + c) * E + e)) : 0;
-        h.super_before[i] = sum;
-    }
-    __syncthreads();
-    // 2. exclusive scan over super-chunks, one thread per expert (loads are independent of the running sum)
-    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) {
-        int running = 0;
-        if (e < E) {
-            for (int sc = 0; sc < h.n_super; ++sc) {
-                const int c = h.super_before[static_cast<size_t>(sc) * E + e];
-                h.super_before[static_cast<size_t>(sc) * E + e] = running;
-                running += c;
-            }
-        }
-        hist[e] = running;
-    }
-    __syncthreads();
-    classify_scan(h, hist);
-}
-
-// Called by every thread of a CTA that has finished a chunk (its top-k stores and its row of chunk
-// counts): the CTA that finishes last runs the tail, so routing is one launch.
-__device__ void finish_route(const HistArgs& h) {
+// Called by every thread of every router CTA after its top-k stores: the CTA that finishes
+// last runs the histogram, so routing is one launch.
+__device__ void finish_route(const HistArgs& h, const int32_t* topk_idx, int finishers = 0) {
     __shared__ int s_hist[kMaxExperts];
     __shared__ int s_last;
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) s_last = atomicAdd(h.ticket, 1) == h.n_chunks - 1;
+    if (finishers == 0) finishers = static_cast<int>(gridDim.x);     // default: every CTA of the launch arrives
+    if (threadIdx.x == 0) s_last = atomicAdd(h.ticket, 1) == finishers - 1;
     __syncthreads();
     if (!s_last) return;
     __threadfence();
     if (threadIdx.x == 0) *h.ticket = 0;
-    histogram_classify_scan(h, s_hist);
-}
-
-// Writes the chunk's row of per-expert counts (called by all threads after a __syncthreads that
-// follows the last softmax_topk_store of the CTA).
-__device__ __forceinline__ void store_chunk_counts(const HistArgs& h, int chunk, const int* chunk_hist) {
-    for (int e = threadIdx.x; e < h.E; e += blockDim.x)
-        h.chunk_counts[static_cast<size_t>(chunk) * h.E + e] = static_cast<uint8_t>(chunk_hist[e]);
+    histogram_classify_scan(h, topk_idx, s_hist);
 }
 
 // Stand-alone form, used when there are no tokens (every count is zero).
-__global__ void __launch_bounds__(256) histogram_only_kernel(HistArgs h) {
+__global__ void __launch_bounds__(256) histogram_only_kernel(HistArgs h, const int32_t* topk_idx) {
     __shared__ int s_hist[kMaxExperts];
     pdl_launch_dependents();
     pdl_wait();
-    histogram_classify_scan(h, s_hist);
+    histogram_classify_scan(h, topk_idx, s_hist);
 }
 
-// One warp per token (16 warps: one chunk per CTA); lanes split d_model with 16-byte loads.
+// One warp per token; lanes split d_model with 16-byte loads.
 template <typename T>
-__global__ void __launch_bounds__(kChunkTokens * 32) route_warp_per_token_kernel(
+__global__ void __launch_bounds__(128) route_warp_per_token_kernel(
         int T_tokens, int d, int E, int k, int renorm, const T* __restrict__ x, const T* __restrict__ Wg,
         const float* __restrict__ bg, int32_t* __restrict__ topk_idx, float* __restrict__ topk_w,
         float* __restrict__ probs, const HistArgs hist) {
     constexpr int V = Vec16<T>::N;
-    __shared__ int s_chunk[kMaxExperts];
     const int lane = threadIdx.x & 31;
-    const int64_t t = static_cast<int64_t>(blockIdx.x) * kChunkTokens + (threadIdx.x >> 5);
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
     pdl_launch_dependents();
-    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) s_chunk[e] = 0;
-    __syncthreads();
     pdl_wait();
     if (t < T_tokens) {
     const T* xr = x + t * d;
@@ -260,11 +229,9 @@ __global__ void __launch_bounds__(kChunkTokens * 32) route_warp_per_token_kernel
             }
         }
     }
-    softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs, s_chunk);
+    softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs);
     }
-    __syncthreads();
-    store_chunk_counts(hist, blockIdx.x, s_chunk);
-    finish_route(hist);
+    finish_route(hist, topk_idx);
 }
 
 // ---- bf16 gate on the warp-level tensor-core path -------------------------------------
@@ -295,13 +262,11 @@ __global__ void __launch_bounds__(512, (kDeep || kTilesPerWarp >= 8) ? 1 : 2) ro
     constexpr int kEPad = 32 * kTilesPerWarp;
     constexpr int kRow = kEPad + 1;
     extern __shared__ float s_part[];                 // [4 K quarters][16 tokens][kRow]
-    __shared__ int s_chunk[kMaxExperts];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int eq = warp & 3, kq = warp >> 2;
     const int g = lane >> 2, t4 = lane & 3;
     const int tok0 = blockIdx.x * 16;
     pdl_launch_dependents();
-    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) s_chunk[e] = 0;
     pdl_wait();
     const int r0 = min(tok0 + g, T_tokens - 1), r1 = min(tok0 + g + 8, T_tokens - 1);
     const uint4* xa = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(r0) * d) + t4;
@@ -320,7 +285,7 @@ __global__ void __launch_bounds__(512, (kDeep || kTilesPerWarp >= 8) ? 1 : 2) ro
     const int steps = d / 32;               // 32 k per step: 4 lanes x 8 elements
     // Loads of several steps are issued together and the MMAs follow: a step at a time would put one
     // trip to memory per step on the critical path of a kernel that is all latency.
-    constexpr int kBatch = kTilesPerWarp >= 8 ? 1 : (kDeep ? 20 / (2 + kTilesPerWarp) : (kTilesPerWarp <= 2 ? 2 : 1));   // loads in flight: about 80 registers (deep), 32 (two CTAs per SM)
+    constexpr int kBatch = (!kDeep || kTilesPerWarp >= 8) ? 1 : 20 / (2 + kTilesPerWarp);   // about 80 registers of loads in flight
     for (int s0 = kq; s0 < steps; s0 += 4 * kBatch) {
         uint4 a[kBatch], b[kBatch], w[kBatch][kTilesPerWarp];
 #pragma unroll
@@ -367,16 +332,14 @@ __global__ void __launch_bounds__(512, (kDeep || kTilesPerWarp >= 8) ? 1 : 2) ro
                 logit[s] = -INFINITY;
             }
         }
-        softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs, s_chunk);
+        softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs);
     }
-    __syncthreads();
-    store_chunk_counts(hist, blockIdx.x, s_chunk);
-    finish_route(hist);
+    finish_route(hist, topk_idx);
 }
 
 // ---- small batches: the gate GEMM dealt over (chunk, 8 experts) CTAs -----------------------------
-// A batch of a few dozen tokens has one or two chunks; with one CTA per chunk a decode step would
-// read the whole gate matrix through one or two SMs.  Here CTA (chunk c, octet o) computes the
+// A batch of a few dozen tokens has one or two 16-token chunks; with one CTA per chunk a decode step
+// would read the whole gate matrix through one or two SMs.  Here CTA (chunk c, octet o) computes the
 // logits of 16 tokens against experts [8o, 8o+8): its 16 warps split K sixteen ways (all loads of
 // the CTA are in flight together: one trip to memory), partial sums meet in shared memory and are
 // added in warp order, and the 16 x 8 logits go to the workspace.  The CTA that completes a chunk's
@@ -387,14 +350,12 @@ __global__ void __launch_bounds__(512, 1) route_split_kernel(
         float* __restrict__ topk_w, float* __restrict__ probs, float* __restrict__ logits_ws,
         int32_t* __restrict__ tile_tickets, const HistArgs hist) {
     __shared__ float s_part[16][16][9];            // [warp][token][expert of the octet]
-    __shared__ int s_chunk[kMaxExperts];
     __shared__ int s_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t4 = lane & 3;
     const int chunk = blockIdx.x, oct = blockIdx.y, n_oct = gridDim.y;
-    const int tok0 = chunk * kChunkTokens;
+    const int tok0 = chunk * 16;
     pdl_launch_dependents();
-    for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) s_chunk[e] = 0;
     pdl_wait();
     const int r0 = min(tok0 + g, T_tokens - 1), r1 = min(tok0 + g + 8, T_tokens - 1);
     const uint4* xa = reinterpret_cast<const uint4*>(x + static_cast<int64_t>(r0) * d) + t4;
@@ -451,11 +412,9 @@ __global__ void __launch_bounds__(512, 1) route_split_kernel(
             const int e = sl * 32 + lane;
             logit[sl] = e < E ? __ldcg(logits_ws + t * kMaxExperts + e) : -INFINITY;
         }
-        softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs, s_chunk);
+        softmax_topk_store(logit, E, k, renorm, t, lane, topk_idx, topk_w, probs);
     }
-    __syncthreads();
-    store_chunk_counts(hist, chunk, s_chunk);
-    finish_route(hist);
+    finish_route(hist, topk_idx, gridDim.x);
 }
 
 template <int kTilesPerWarp>
@@ -550,22 +509,19 @@ __global__ void __launch_bounds__(kMaxExperts) classify_top_h_kernel(
 int launch_route(const monde_problem& p, const void* x, const void* Wg, const float* bg,
                  int32_t* topk_idx, float* topk_w, float* probs, int32_t* counts, int32_t* offsets, uint8_t* cls,
                  int32_t* hot_ids, int32_t* cold_ids, int32_t* n_hot_cold, void* ws, cudaStream_t s) {
-    const WsLayout L = ws_layout(p);
     char* base = static_cast<char*>(ws);
     int32_t* ticket = reinterpret_cast<int32_t*>(base + WsLayout::kRouteTicket);
-    const HistArgs hist{p.T, p.E, p.hot_threshold, L.n_chunks, L.n_super, counts, offsets, cls, hot_ids, cold_ids,
-                        n_hot_cold, ticket, reinterpret_cast<uint8_t*>(base + L.chunk_counts_off),
-                        reinterpret_cast<int32_t*>(base + L.super_before_off)};
+    const HistArgs hist{p.T * p.top_k, p.E, p.hot_threshold, counts, offsets, cls, hot_ids, cold_ids, n_hot_cold, ticket};
     if (p.T == 0) {
-        launch_pdl(histogram_only_kernel, dim3(1), dim3(256), 0, s, hist);
+        launch_pdl(histogram_only_kernel, dim3(1), dim3(256), 0, s, hist, topk_idx);
         return launched();
     }
     if (p.dtype == MONDE_BF16 && p.T <= kSplitRouteMaxTokens) {
         // at most 16 chunks: their tickets follow the call's own in the workspace header
-        launch_pdl(route_split_kernel, dim3(L.n_chunks, (p.E + 7) / 8), dim3(512), 0, s,
+        launch_pdl(route_split_kernel, dim3((p.T + 15) / 16, (p.E + 7) / 8), dim3(512), 0, s,
             p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const __nv_bfloat16*>(x),
             static_cast<const __nv_bfloat16*>(Wg), bg, topk_idx, topk_w, probs,
-            reinterpret_cast<float*>(base + L.logits_off), ticket + 1, hist);
+            reinterpret_cast<float*>(base + ws_layout(p).logits_off), ticket + 1, hist);
         return launched();
     }
     if (p.dtype == MONDE_BF16) {
@@ -576,7 +532,8 @@ int launch_route(const monde_problem& p, const void* x, const void* Wg, const fl
         else st = launch_route_mma<8>(p, x, Wg, bg, topk_idx, topk_w, probs, hist, s);
         if (st != MONDE_OK) return st;
     } else {
-        launch_pdl(route_warp_per_token_kernel<float>, dim3(L.n_chunks), dim3(kChunkTokens * 32), 0, s,
+        const int warps = 4;
+        launch_pdl(route_warp_per_token_kernel<float>, dim3((p.T + warps - 1) / warps), dim3(warps * 32), 0, s,
             p.T, p.d_model, p.E, p.top_k, p.renormalize, static_cast<const float*>(x),
             static_cast<const float*>(Wg), bg, topk_idx, topk_w, probs, hist);
     }

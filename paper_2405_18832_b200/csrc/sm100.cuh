@@ -113,92 +113,43 @@ __device__ __forceinline__ void tc_fence_before_sync() {
 __device__ __forceinline__ void tc_fence_after_sync() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
-// One whole 64-wide K block of a unit as a single instruction sequence: the probes of the next
-// stage's "full" barriers are issued first, then the 4 MMAs of each of the unit's feature tiles
-// (second tile: operand A 16 KB further on, accumulator d1), then the commits that hand the stage
-// back to the producers, and the probe answers are read last.  The issuing thread is held by each
-// MMA until the tensor pipe accepts it, so everything whose latency can overlap the pipe's work
-// (probe round trips, commits) is placed behind the MMAs instead of in front of them.
-// kTiles: 1 or 2 feature tiles.  kBars: 2 = separate weight / token rings (two probes, two commits),
-// 1 = one barrier pair serves both rings (probe_b / commit_b unused).
-// Returns true when every probed phase is complete.
-template <int kTiles, int kBars>
-__device__ __forceinline__ bool umma_bf16_kblock(uint32_t d0, uint32_t d1, uint64_t a_desc, uint64_t b_desc,
-                                                 uint32_t idesc, uint32_t accumulate, uint32_t probe_a,
-                                                 uint32_t parity_a, uint32_t probe_b, uint32_t parity_b,
-                                                 uint32_t commit_a, uint32_t commit_b) {
+// D[tmem] (+)= A[smem] * B[smem]; one thread issues.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) );
+}
+// Four MMAs over one 64-wide K block (descriptors advance by 32 bytes per 16 columns) with a
+// non-blocking probe of two mbarriers issued first and read last: the probes take over a
+// hundred cycles to answer, and the issuing thread would otherwise sit out that time before
+// every K block.  `accumulate` applies to the first MMA; the other three always accumulate.
+// Returns true when both probed phases are complete.
+__device__ __forceinline__ bool umma_bf16_x4_probe(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                   uint32_t accumulate, uint32_t bar_a, uint32_t parity_a,
+                                                   uint32_t bar_b, uint32_t parity_b) {
     uint32_t ready;
-#define MONDE_MMA4(D, A0, PFIRST)                                                           \
-        "add.s64 a, %3, " A0 ";\n\t"                                                         \
-        "tcgen05.mma.cta_group::1.kind::f16 [" D "], a, %4, %5, " PFIRST ";\n\t"             \
-        "add.s64 a, a, 2;\n\tadd.s64 b, %4, 2;\n\t"                                         \
-        "tcgen05.mma.cta_group::1.kind::f16 [" D "], a, b, %5, t;\n\t"                       \
-        "add.s64 a, a, 2;\n\tadd.s64 b, %4, 4;\n\t"                                         \
-        "tcgen05.mma.cta_group::1.kind::f16 [" D "], a, b, %5, t;\n\t"                       \
-        "add.s64 a, a, 2;\n\tadd.s64 b, %4, 6;\n\t"                                         \
-        "tcgen05.mma.cta_group::1.kind::f16 [" D "], a, b, %5, t;\n\t"
-    if (kTiles == 2 && kBars == 2) {
-        asm volatile(
-            "{\n\t.reg .pred pa, pb, p, t;\n\t.reg .b64 a, b;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 pa, [%7], %8;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 pb, [%9], %10;\n\t"
-            "setp.ne.b32 p, %6, 0;\n\t"
-            "setp.eq.b32 t, 0, 0;\n\t"
-            MONDE_MMA4("%1", "0", "p")
-            MONDE_MMA4("%2", "1024", "p")
-            "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%11];\n\t"
-            "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%12];\n\t"
-            "and.pred pa, pa, pb;\n\t"
-            "selp.u32 %0, 1, 0, pa;\n\t}"
-            : "=r"(ready)
-            : "r"(d0), "r"(d1), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(probe_a), "r"(parity_a),
-              "r"(probe_b), "r"(parity_b), "r"(commit_a), "r"(commit_b)
-            : "memory");
-    } else if (kTiles == 1 && kBars == 2) {
-        asm volatile(
-            "{\n\t.reg .pred pa, pb, p, t;\n\t.reg .b64 a, b;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 pa, [%7], %8;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 pb, [%9], %10;\n\t"
-            "setp.ne.b32 p, %6, 0;\n\t"
-            "setp.eq.b32 t, 0, 0;\n\t"
-            MONDE_MMA4("%1", "0", "p")
-            "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%11];\n\t"
-            "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%12];\n\t"
-            "and.pred pa, pa, pb;\n\t"
-            "selp.u32 %0, 1, 0, pa;\n\t}"
-            : "=r"(ready)
-            : "r"(d0), "r"(d1), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(probe_a), "r"(parity_a),
-              "r"(probe_b), "r"(parity_b), "r"(commit_a), "r"(commit_b)
-            : "memory");
-    } else if (kTiles == 2) {
-        asm volatile(
-            "{\n\t.reg .pred pa, p, t;\n\t.reg .b64 a, b;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 pa, [%7], %8;\n\t"
-            "setp.ne.b32 p, %6, 0;\n\t"
-            "setp.eq.b32 t, 0, 0;\n\t"
-            MONDE_MMA4("%1", "0", "p")
-            MONDE_MMA4("%2", "1024", "p")
-            "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n\t"
-            "selp.u32 %0, 1, 0, pa;\n\t}"
-            : "=r"(ready)
-            : "r"(d0), "r"(d1), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(probe_a), "r"(parity_a),
-              "r"(commit_a)
-            : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred pa, p, t;\n\t.reg .b64 a, b;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 pa, [%7], %8;\n\t"
-            "setp.ne.b32 p, %6, 0;\n\t"
-            "setp.eq.b32 t, 0, 0;\n\t"
-            MONDE_MMA4("%1", "0", "p")
-            "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n\t"
-            "selp.u32 %0, 1, 0, pa;\n\t}"
-            : "=r"(ready)
-            : "r"(d0), "r"(d1), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(probe_a), "r"(parity_a),
-              "r"(commit_a)
-            : "memory");
-    }
-#undef MONDE_MMA4
+    asm volatile(
+        "{\n\t.reg .pred pa, pb, p, t;\n\t.reg .b64 a, b;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 pa, [%6], %7;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 pb, [%8], %9;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "setp.eq.b32 t, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t"
+        "add.s64 a, %2, 2;\n\tadd.s64 b, %3, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], a, b, %4, t;\n\t"
+        "add.s64 a, %2, 4;\n\tadd.s64 b, %3, 4;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], a, b, %4, t;\n\t"
+        "add.s64 a, %2, 6;\n\tadd.s64 b, %3, 6;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%1], a, b, %4, t;\n\t"
+        "and.pred pa, pa, pb;\n\t"
+        "selp.u32 %0, 1, 0, pa;\n\t}"
+        : "=r"(ready)
+        : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(bar_a), "r"(parity_a), "r"(bar_b),
+          "r"(parity_b)
+        : "memory");
     return ready != 0;
 }
 // Arrives on `bar` once every tcgen05.mma issued so far by this thread has completed.
