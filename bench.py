@@ -230,6 +230,15 @@ def workload_config(w):
             "parallelism": "independent replicas, one per GPU, no data-path collective"}
 
 
+def use_fused_combine(args, p) -> bool:
+    """The layer is timed in the faster of its two bit-identical forms: FFN + combine in one call where that
+    wins (top-1 routing, bf16: `binding.fused_combine_wins`), four calls otherwise; the flags force either."""
+    from paper_2405_18832_b200 import binding as B
+    if p.dtype != "bf16" or args.no_fuse_combine:
+        return False
+    return True if args.fuse_combine else B.fused_combine_wins(p)
+
+
 def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline, weights=None, light=False):
     """All measurements of one workload on this rank's GPU; returns the result record (rank 0) or None.
     `weights`: expert weights already on the device (same seed and shapes), `light`: no host-buffer runs."""
@@ -248,7 +257,7 @@ def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline, weights=N
     L = B.lib()
     warmup = max(args.warmup, 3)
 
-    fuse = bool(args.fuse_combine) and p.dtype == "bf16"
+    fuse = use_fused_combine(args, p)
 
     def layer(ev=None):
         if ev is not None:
@@ -343,7 +352,7 @@ def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline, weights=N
 
     e2e = None
     if not light:
-        e2e = measure_host_buffers(B, p, g, d, buf, flush, stream, steps, warmup, dist, dev, world)
+        e2e = measure_host_buffers(B, p, g, d, buf, flush, stream, steps, warmup, dist, dev, world, fuse)
     del flush
 
     if rank != 0:
@@ -354,7 +363,7 @@ def measure(args, w, dist, rank, world, dev, steps, with_cpu_baseline, weights=N
     return rec
 
 
-def measure_host_buffers(B, p, g, d, buf, flush, stream, steps, warmup, dist, dev, world):
+def measure_host_buffers(B, p, g, d, buf, flush, stream, steps, warmup, dist, dev, world, fuse):
     # ---- end to end: tokens in pinned host memory ----------------------------------
     # Every step copies its tokens host -> device and its result device -> host.  Serial form:
     # copy, four calls, copy, wait (per-step latency).  Pipelined form (the e2e figure): the same
@@ -364,20 +373,22 @@ def measure_host_buffers(B, p, g, d, buf, flush, stream, steps, warmup, dist, de
     x_host = g["x"].pin_memory()
     out_host = torch.empty((p.T, p.d_model), dtype=p.torch_dtype).pin_memory()
     for _ in range(3):
-        B.moe_ffn_layer_forward_host(p, x_host, out_host, d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"], buf)
+        B.moe_ffn_layer_forward_host(p, x_host, out_host, d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"], buf,
+                                     fuse_combine=fuse)
     e2e_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     torch.cuda.synchronize()
     for a, b in e2e_ev:
         flush.fill_(3)
         a.record(stream)
-        B.moe_ffn_layer_forward_host(p, x_host, out_host, d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"], buf)
+        B.moe_ffn_layer_forward_host(p, x_host, out_host, d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"], buf,
+                                     fuse_combine=fuse)
         b.record(stream)
     torch.cuda.synchronize()
     serial_ms = max_over_ranks(dist, sum(a.elapsed_time(b) for a, b in e2e_ev), dev)
     e2e_serial_value = aggregate_tokens_per_s(p.T, world, serial_ms / steps)
     assert torch.equal(out_host, buf.out.cpu())
 
-    pipe = B.HostPipeline(p, depth=2, device=dev)
+    pipe = B.HostPipeline(p, depth=2, device=dev, fuse_combine=fuse)
     weights = (d["Wg"], d["bg"], d["W1"], d["b1"], d["W2"], d["b2"])
     out_host.zero_()
     for _ in range(warmup):
@@ -405,7 +416,7 @@ def measure_host_buffers(B, p, g, d, buf, flush, stream, steps, warmup, dist, de
 
 def summarise(args, w, p, counts, n_hot_used, steps, warmup, world, ms_per_step, step_ms, call_ms, value, clocks, launches,
               wall, e2e, g, with_cpu_baseline):
-    fuse = bool(args.fuse_combine) and p.dtype == "bf16"
+    fuse = use_fused_combine(args, p)
     peaks = measured_peaks()
     ffn_ms = statistics.mean(call_ms[2])
     bytes_ffn = ffn_algorithmic_bytes(p, counts)
@@ -413,7 +424,9 @@ def summarise(args, w, p, counts, n_hot_used, steps, warmup, world, ms_per_step,
     tflops = ffn_flops(p, counts) / (ffn_ms * 1e-3) / 1e12
     traffic, traffic_source = NCU_TRAFFIC.get(w.name, (None, "no capture for this workload"))
     tensor_bound = w.name == "HOTPROBE"      # the one workload whose experts sit far above the ridge
-    common = {"kernel": "expert_ffn_kernel via monde_moe_ffn_fwd (hot + cold expert FFN, both layers)",
+    common = {"kernel": "expert_ffn_kernel via " + ("monde_moe_ffn_combine_fwd (hot + cold expert FFN, both layers, gate "
+                                                    "weight applied in the last store)" if fuse else
+                                                    "monde_moe_ffn_fwd (hot + cold expert FFN, both layers)"),
               "peak_source": peaks["source"], "traffic": traffic, "traffic_source": traffic_source,
               "algorithmic_bytes": bytes_ffn, "algorithmic_flops": ffn_flops(p, counts), "ms": ffn_ms,
               "units_per_launch": int((counts > 0).sum()), "unit": "GB/s",
@@ -465,8 +478,8 @@ def summarise(args, w, p, counts, n_hot_used, steps, warmup, world, ms_per_step,
         "gpu_launches": launches,
         "roofline": roofline, "cpu_baseline": cpu,
         "calls_ms": {"route": statistics.mean(call_ms[0]), "permute": statistics.mean(call_ms[1]),
-                     "ffn": ffn_ms, "combine": statistics.mean(call_ms[3])},
-        "calls_ms_sum": sum(statistics.mean(c) for c in call_ms),
+                     "ffn": ffn_ms, "combine": 0.0 if fuse else statistics.mean(call_ms[3])},
+        "calls_ms_sum": sum(statistics.mean(c) for c in call_ms[:3 if fuse else 4]),
         "layer_hbm_floor_ms": layer_floor_ms, "layer_roofline_frac": layer_floor_ms / ms_per_step,
         "layer_lower_bound": {"formula": "sum over activated experts of max(flops / tensor peak, bytes / HBM peak) "
                                          "+ elementwise bytes / HBM peak",
@@ -484,7 +497,7 @@ def summarise(args, w, p, counts, n_hot_used, steps, warmup, world, ms_per_step,
 
 SUB_WORKLOADS = ("C2", "C1", "HOTPROBE")
 SUB_KEYS = ("value", "unit", "steps", "ms_per_step", "config", "clocks", "e2e", "roofline", "calls_ms", "calls_ms_sum",
-            "layer_lower_bound", "layer_roofline_frac", "step_ms", "routing", "gpu_launches")
+            "layer_lower_bound", "layer_roofline_frac", "step_ms", "routing", "gpu_launches", "calls")
 
 
 def sub_steps(name: str, steps: int) -> int:
@@ -583,7 +596,9 @@ def main():
                     help="run the 90-point crossover sweep (resumable) instead of a single workload")
     ap.add_argument("--sweep-out", default=os.path.join(ROOT, "gpurun_out", "sweep_C4.jsonl"))
     ap.add_argument("--fuse-combine", action="store_true",
-                    help="bf16 workloads: monde_moe_ffn_combine_fwd instead of monde_moe_ffn_fwd + monde_combine")
+                    help="bf16 workloads: always monde_moe_ffn_combine_fwd (default: where it is the faster form, top-1)")
+    ap.add_argument("--no-fuse-combine", action="store_true",
+                    help="always the four-call form: monde_moe_ffn_fwd + monde_combine")
     ap.add_argument("--policy", default="threshold", choices=["threshold", "top_h"],
                     help="hot/cold rule: count >= hot_threshold, or the paper's top-H rule (Eq. 6)")
     ap.add_argument("--alpha", type=float, default=1.0, help="Eq. 6 tuning factor (top_h)")

@@ -249,12 +249,20 @@ def moe_ffn_layer_forward(p, x, Wg, bg, W1, b1, W2, b2, buf: LayerBuffers, strea
     return buf.out
 
 
+def fused_combine_wins(p) -> bool:
+    """Whether monde_moe_ffn_combine_fwd is the faster of the two bit-identical forms of the layer: measured,
+    it saves the combine kernel for top-1 routing (2-4 us per layer) and costs time for top-k > 1, where the
+    staging rows are written and read like y_perm."""
+    cp = c_problem(p)
+    return cp.top_k == 1 and cp.dtype == 1
+
+
 def moe_ffn_layer_forward_host(p, x_host, out_host, Wg, bg, W1, b1, W2, b2, buf: LayerBuffers,
-                               stream=None) -> torch.Tensor:
+                               stream=None, fuse_combine: bool = False) -> torch.Tensor:
     """Same layer with the step's tokens in pinned host memory: copies them to the device,
     runs the layer, copies the result back and waits for it."""
     buf.x_dev.copy_(x_host, non_blocking=True)
-    out = moe_ffn_layer_forward(p, buf.x_dev, Wg, bg, W1, b1, W2, b2, buf, stream)
+    out = moe_ffn_layer_forward(p, buf.x_dev, Wg, bg, W1, b1, W2, b2, buf, stream, fuse_combine)
     out_host.copy_(out, non_blocking=True)
     (torch.cuda.current_stream() if stream is None else stream).synchronize()
     return out_host
@@ -270,9 +278,10 @@ class HostPipeline:
     steps differs from `moe_ffn_layer_forward_host`.
     """
 
-    def __init__(self, p, depth: int = 2, device="cuda"):
+    def __init__(self, p, depth: int = 2, device="cuda", fuse_combine: bool = False):
         self.p = p
         self.depth = depth
+        self.fuse_combine = fuse_combine
         self.bufs = [LayerBuffers(p, device=device) for _ in range(depth)]
         self.s_in = torch.cuda.Stream(device=device)
         self.s_run = torch.cuda.Stream(device=device)
@@ -295,7 +304,7 @@ class HostPipeline:
         self.s_run.wait_event(self.copied_in[i])
         if reused:
             self.s_run.wait_event(self.copied_out[i])     # this buffer set's previous result has left
-        moe_ffn_layer_forward(self.p, buf.x_dev, Wg, bg, W1, b1, W2, b2, buf, self.s_run)
+        moe_ffn_layer_forward(self.p, buf.x_dev, Wg, bg, W1, b1, W2, b2, buf, self.s_run, self.fuse_combine)
         self.computed[i].record(self.s_run)
         self.s_out.wait_event(self.computed[i])
         with torch.cuda.stream(self.s_out):
