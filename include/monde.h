@@ -50,7 +50,8 @@ typedef enum {
     MONDE_ERR_WORKSPACE = 3,    /* ws_bytes smaller than monde_workspace_bytes() */
     MONDE_ERR_ARCH = 4,         /* current device is not compute capability 10.x */
     MONDE_ERR_CUDA = 5,         /* a CUDA runtime / driver call failed */
-    MONDE_ERR_TIMEOUT = 6       /* a bounded device-side wait gave up */
+    MONDE_ERR_TIMEOUT = 6,      /* a bounded device-side wait gave up */
+    MONDE_ERR_BOUNDS = 7        /* diagnostics build only: an index read from memory was out of range */
 } monde_status;
 
 typedef enum { MONDE_F32 = 0, MONDE_BF16 = 1 } monde_dtype;

@@ -9,6 +9,8 @@
 #ifndef MONDE_DIAGNOSTICS_H_
 #define MONDE_DIAGNOSTICS_H_
 
+#include <stdint.h>
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -41,6 +43,18 @@ void monde_diag_set_hold_hidden_ready(int on);
  * have run on CUDA device `device` in this process: they run once per device, with that device
  * current, at the first call that needs them.  -1 for a device index outside 0..63. */
 int monde_diag_device_setups(int device);
+
+/* Range checks.  A library built with -DMONDE_DIAGNOSTICS (`python -m paper_2405_18832_b200.build
+ * --diagnostics` makes libmonde_diag.so) checks every index its kernels take from memory before using
+ * it as an address: expert ids and positions in the permutation, positions in the combine, the rows
+ * and features of every work unit of the expert FFN.  A value out of range is counted, the first one
+ * is kept with a site code (1 permute expert id, 2 permute position, 3 combine position, 4 FFN unit
+ * rows, 5 FFN unit features), and the access is skipped; an FFN unit out of range also records
+ * MONDE_ERR_BOUNDS in the workspace.  It stands in for a memory checker where none may be run.
+ * This call synchronises the device, returns the number of violations since the last call and
+ * clears the record; `first_site` / `first_value` (nullable, host pointers) receive the first one.
+ * Returns -1 from a library that was not built with the checks, -2 if the record cannot be read. */
+int monde_diag_bounds_violations(int32_t* first_site, long long* first_value);
 
 #ifdef __cplusplus
 }

@@ -20,7 +20,7 @@ SYMBOLS = ("monde_workspace_bytes", "monde_status_string", "monde_route", "monde
            "monde_moe_ffn_fwd", "monde_moe_ffn_combine_fwd", "monde_moe_ffn_fwd_static_ws", "monde_combine", "monde_poll_device_status",
            "monde_kernel_launches", "monde_poll_static_ws_status",
            "monde_diag_set_ffn_cta_pairs", "monde_diag_set_trace", "monde_diag_set_wait_limit_ns",
-           "monde_diag_set_hold_hidden_ready", "monde_diag_device_setups")
+           "monde_diag_set_hold_hidden_ready", "monde_diag_device_setups", "monde_diag_bounds_violations")
 
 _DTYPE = {"f32": 0, "bf16": 1}
 _ACT = {"relu": 0, "gelu": 1}
@@ -89,6 +89,8 @@ def lib() -> ctypes.CDLL:
         L.monde_diag_set_hold_hidden_ready.argtypes = [ctypes.c_int]
         L.monde_diag_device_setups.restype = ctypes.c_int
         L.monde_diag_device_setups.argtypes = [ctypes.c_int]
+        L.monde_diag_bounds_violations.restype = ctypes.c_int
+        L.monde_diag_bounds_violations.argtypes = [ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_longlong)]
         _lib = L
     return _lib
 

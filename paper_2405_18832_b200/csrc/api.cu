@@ -67,6 +67,26 @@ std::atomic<unsigned long long> g_wait_limit_ns{kDefaultWaitLimitNs};
 std::atomic<int> g_hold_hidden_ready{0};
 }  // namespace
 
+#ifdef MONDE_DIAGNOSTICS
+namespace {
+__device__ DiagRecord g_diag_record;      // host code may only take its address through cudaGetSymbolAddress
+DiagRecord* g_diag_ptr[kMaxDevices] = {};
+}  // namespace
+DiagRecord* diag_record_ptr() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (g_diag_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_diag_record) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        g_diag_ptr[dev] = static_cast<DiagRecord*>(p);
+    }
+    return g_diag_ptr[dev];
+}
+#else
+DiagRecord* diag_record_ptr() { return nullptr; }
+#endif
+
 DiagState diag_state() {
     DiagState d;
     d.trace = g_trace.load(std::memory_order_relaxed);
@@ -128,6 +148,7 @@ const char* monde_status_string(int status) {
         case MONDE_ERR_ARCH: return "device is not compute capability 10.x";
         case MONDE_ERR_CUDA: return "CUDA call failed";
         case MONDE_ERR_TIMEOUT: return "device-side wait timed out";
+        case MONDE_ERR_BOUNDS: return "index out of range (diagnostics build)";
         default: return "unknown status";
     }
 }
@@ -262,6 +283,25 @@ int monde_poll_device_status(void* ws, void* stream, int32_t* site) {
 }
 
 // ---- include/monde_diagnostics.h --------------------------------------------------------------
+int monde_diag_bounds_violations(int32_t* first_site, long long* first_value) {
+#ifdef MONDE_DIAGNOSTICS
+    DiagRecord* dev = diag_record_ptr();
+    if (dev == nullptr) return -2;
+    DiagRecord rec;
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy(&rec, dev, sizeof rec, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemset(dev, 0, sizeof rec) != cudaSuccess)
+        return -2;
+    if (first_site != nullptr) *first_site = rec.site;
+    if (first_value != nullptr) *first_value = rec.value;
+    return rec.count;
+#else
+    (void)first_site;
+    (void)first_value;
+    return -1;      // not a diagnostics build
+#endif
+}
+
 void monde_diag_set_ffn_cta_pairs(int mode) { g_ffn_pair.store(mode < 0 ? -1 : (mode != 0), std::memory_order_relaxed); }
 
 void monde_diag_set_trace(void* device_buf, int slots) {

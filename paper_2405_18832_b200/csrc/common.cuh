@@ -167,6 +167,31 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
 // Process-wide count of kernels this library has launched (diagnostic).
 void count_launches(int n);
 
+// ---- range checks of the diagnostics build ---------------------------------------------------
+// Built with -DMONDE_DIAGNOSTICS the kernels check every index they take from memory before they use
+// it as an address (expert ids, positions of the permutation, the rows and features of an FFN work
+// unit), count violations in a record inside the library's device image, keep the first one (site and
+// value) and skip the access.  The ordinary build compiles the checks away.  This stands in for a
+// memory checker on machines where none may be run.
+struct DiagRecord {
+    int32_t count;      // violations since the record was last read
+    int32_t site;       // of the first one: 1 permute expert id, 2 permute position, 3 combine position,
+    long long value;    //                   4 FFN unit rows, 5 FFN unit features; and the offending value
+};
+DiagRecord* diag_record_ptr();    // device address of the record on the current device; null in the ordinary build
+#ifdef MONDE_DIAGNOSTICS
+__device__ __forceinline__ bool diag_in_range(bool ok, DiagRecord* rec, int site, long long value) {
+    if (!ok && rec != nullptr && atomicAdd(&rec->count, 1) == 0) {
+        rec->site = site;
+        rec->value = value;
+    }
+    return ok;
+}
+#define MONDE_IN_RANGE(cond, rec, site, value) diag_in_range((cond), (rec), (site), static_cast<long long>(value))
+#else
+#define MONDE_IN_RANGE(cond, rec, site, value) true
+#endif
+
 // ---- per-device set-up ---------------------------------------------------------------------
 // Function attributes (the opt-in to more than 48 KB of dynamic shared memory) and the SM count
 // belong to a device, not to the process: a process that drives several GPUs must set them up on

@@ -104,6 +104,8 @@ struct FfnParams {
     const int32_t* fuse_perm;    // fused combine: assignment id of every row; null = store y in expert-contiguous order
     const float* fuse_w;         // gate weight per assignment (top-1); null = rows go out unweighted, in assignment order
     __nv_bfloat16* fuse_out;     // out [T, d_model] (top-1) or the token-ordered staging rows [T * top_k, d_model]
+    DiagRecord* diag;            // range-check record of the diagnostics build (null otherwise)
+    int A;                       // rows of x_perm / h / y_perm
     unsigned long long* trace;   // diagnostic timeline (null in normal use): [cta][unit slot][8]
     int trace_slots;
     int hold_ready;              // diagnostic: first-layer units do not publish their rows
@@ -583,10 +585,22 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                 }
                 return mail[slot];
             };
+            // Diagnostics build: a decoded unit whose rows or features fall outside the problem is recorded
+            // and ends this CTA's list (nothing of it is loaded or stored).
+            auto checked = [&](Unit un) -> Unit {
+                [[maybe_unused]] const int N = un.layer ? P.d_model : P.d_ff;
+                if (!MONDE_IN_RANGE(un.row0 >= 0 && un.rows > 0 && un.row0 + un.rows <= P.A, P.diag, 4, un.row0) ||
+                    !MONDE_IN_RANGE(un.e >= 0 && un.e < P.E && un.n0 >= 0 && un.n0 < N && un.kb0 >= 0 && un.kb0 < un.kb1,
+                                    P.diag, 5, un.n0)) {
+                    if (atomicCAS(P.status, 0, MONDE_ERR_BOUNDS) == 0) P.status[1] = un.id;
+                    un.id = -1;
+                }
+                return un;
+            };
             Unit cur, nxt;
             const int u = take_next();
             cur.id = -1;
-            if (u < ut.total_units) cur = ut.decode(u);
+            if (u < ut.total_units) cur = checked(ut.decode(u));
             ok = push_unit(0, cur);
             int u_ahead = cur.id >= 0 ? take_next() : 0;   // used a few K blocks later
             for (int it = 0; ok && cur.id >= 0; ++it) {
@@ -622,7 +636,7 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
                         // the whole of it while other SMs run out of units of its kind)
                         nxt.id = -1;
                         if (u_ahead < ut.total_units) {
-                            nxt = ut.decode(u_ahead);
+                            nxt = checked(ut.decode(u_ahead));
                             u_ahead = take_next();
                         }
                         if (!push_unit(it + 1, nxt)) { ok = false; break; }
@@ -1238,6 +1252,8 @@ int launch_ffn_bf16(const monde_problem& p, const void* x_perm, const void* W1, 
     P.fuse_perm = fuse_perm;
     P.fuse_w = fuse_w;
     P.fuse_out = static_cast<__nv_bfloat16*>(fuse_out);
+    P.diag = diag_record_ptr();
+    P.A = static_cast<int>(A);
     P.trace = diag.trace;
     P.trace_slots = diag.trace_slots;
     P.hold_ready = diag.hold_hidden_ready;

@@ -25,14 +25,17 @@ constexpr int kSuper = 2048;         // assignments per super-chunk
 constexpr int kTwoLevelFrom = 8192;  // batches with more assignments take the two-level path
 
 __global__ void __launch_bounds__(256) super_histogram_kernel(int A, int E, const int32_t* __restrict__ topk_idx,
-                                                              int32_t* __restrict__ super_before) {
+                                                              int32_t* __restrict__ super_before, DiagRecord* diag) {
     __shared__ int hist[kMaxExperts];
     pdl_launch_dependents();
     for (int e = threadIdx.x; e < kMaxExperts; e += blockDim.x) hist[e] = 0;
     __syncthreads();
     pdl_wait();
     const int first = blockIdx.x * kSuper;
-    for (int a = first + threadIdx.x; a < min(A, first + kSuper); a += blockDim.x) atomicAdd(&hist[topk_idx[a]], 1);
+    for (int a = first + threadIdx.x; a < min(A, first + kSuper); a += blockDim.x) {
+        const int e = topk_idx[a];
+        if (MONDE_IN_RANGE(e >= 0 && e < E, diag, 1, e)) atomicAdd(&hist[e], 1);
+    }
     __syncthreads();
     for (int e = threadIdx.x; e < E; e += blockDim.x) super_before[static_cast<size_t>(blockIdx.x) * E + e] = hist[e];
 }
@@ -55,7 +58,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
         int A, int E, int k, int d, const T* __restrict__ x, const int32_t* __restrict__ topk_idx,
         const int32_t* __restrict__ offsets, const int32_t* __restrict__ super_before,
-        int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, T* __restrict__ x_perm) {
+        int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm, T* __restrict__ x_perm, DiagRecord* diag) {
     __shared__ int before[kMaxExperts];   // assignments to e in earlier chunks
     __shared__ int row_pos[kChunk];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -101,25 +104,33 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 if (v[j].x < 0) continue;
-                atomicAdd(&before[v[j].x], 1);
-                atomicAdd(&before[v[j].y], 1);
-                atomicAdd(&before[v[j].z], 1);
-                atomicAdd(&before[v[j].w], 1);
+                const int ev[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (MONDE_IN_RANGE(ev[i] >= 0 && ev[i] < E, diag, 1, ev[i])) atomicAdd(&before[ev[i]], 1);
             }
         }
     } else {
-        for (int a = recount_from + tid; a < first; a += kThreads) atomicAdd(&before[topk_idx[a]], 1);
+        for (int a = recount_from + tid; a < first; a += kThreads) {
+            const int e = topk_idx[a];
+            if (MONDE_IN_RANGE(e >= 0 && e < E, diag, 1, e)) atomicAdd(&before[e], 1);
+        }
     }
     __syncthreads();
     if (warp == 0) {
         const int a = first + lane;
-        const int e = (lane < kChunk && a < A) ? topk_idx[a] : -1;
+        int e = (lane < kChunk && a < A) ? topk_idx[a] : -1;
+        if (e >= 0 && !MONDE_IN_RANGE(e < E, diag, 1, e)) e = -1;
         const unsigned same = __match_any_sync(0xffffffffu, e);
         int pos = -1;
         if (e >= 0) {
             pos = offsets[e] + before[e] + __popc(same & ((1u << lane) - 1u));
-            perm[pos] = a;
-            inv_perm[a] = pos;
+            if (MONDE_IN_RANGE(pos >= 0 && pos < A, diag, 2, pos)) {
+                perm[pos] = a;
+                inv_perm[a] = pos;
+            } else {
+                pos = -1;
+            }
         }
         if (lane < kChunk) row_pos[lane] = pos;
     }
@@ -152,7 +163,7 @@ __global__ void __launch_bounds__(kThreads) permute_gather_kernel(
 template <typename T>
 __global__ void __launch_bounds__(256) combine_kernel(
         int T_tokens, int d, int k, const T* __restrict__ y_perm, const int32_t* __restrict__ inv_perm,
-        const float* __restrict__ topk_w, T* __restrict__ out) {
+        const float* __restrict__ topk_w, T* __restrict__ out, DiagRecord* diag) {
     constexpr int V = Vec16<T>::N;
     const int vec_per_row = d / V;
     const int64_t g = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -167,6 +178,7 @@ __global__ void __launch_bounds__(256) combine_kernel(
     for (int j = 0; j < k; ++j) {
         const int pos = inv_perm != nullptr ? inv_perm[t * k + j] : static_cast<int>(t * k + j);   // null: rows already in token order
         const float w = topk_w[t * k + j];
+        if (!MONDE_IN_RANGE(pos >= 0 && pos < T_tokens * k, diag, 3, pos)) continue;
         float y[V];
         Vec16<T>::load(y_perm + static_cast<int64_t>(pos) * d + c, y);
 #pragma unroll
@@ -188,18 +200,19 @@ int launch_permute(const monde_problem& p, const void* x, const int32_t* topk_id
     if (A > kTwoLevelFrom) {
         const int n_super = (A + kSuper - 1) / kSuper;
         super_before = scratch;      // n_super * E int32
-        launch_pdl(super_histogram_kernel, dim3(n_super), dim3(256), 0, s, A, p.E, topk_idx, super_before);
+        launch_pdl(super_histogram_kernel, dim3(n_super), dim3(256), 0, s, A, p.E, topk_idx, super_before,
+                   diag_record_ptr());
         launch_pdl(super_scan_kernel, dim3(1), dim3(256), 0, s, n_super, p.E, super_before);
         count_launches(2);
     }
     if (p.dtype == MONDE_BF16)
         launch_pdl(permute_gather_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), 0, s,
             A, p.E, p.top_k, p.d_model, static_cast<const __nv_bfloat16*>(x), topk_idx, offsets, super_before, perm,
-            inv_perm, static_cast<__nv_bfloat16*>(x_perm));
+            inv_perm, static_cast<__nv_bfloat16*>(x_perm), diag_record_ptr());
     else
         launch_pdl(permute_gather_kernel<float>, dim3(grid), dim3(kThreads), 0, s,
             A, p.E, p.top_k, p.d_model, static_cast<const float*>(x), topk_idx, offsets, super_before, perm, inv_perm,
-            static_cast<float*>(x_perm));
+            static_cast<float*>(x_perm), diag_record_ptr());
     return launched();
 }
 
@@ -211,10 +224,10 @@ int launch_combine(const monde_problem& p, const void* y_perm, const int32_t* in
     if (p.dtype == MONDE_BF16)
         launch_pdl(combine_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, s,
             p.T, p.d_model, p.top_k, static_cast<const __nv_bfloat16*>(y_perm), inv_perm, topk_w,
-            static_cast<__nv_bfloat16*>(out));
+            static_cast<__nv_bfloat16*>(out), diag_record_ptr());
     else
         launch_pdl(combine_kernel<float>, dim3(grid), dim3(256), 0, s, p.T, p.d_model, p.top_k, static_cast<const float*>(y_perm),
-                                                   inv_perm, topk_w, static_cast<float*>(out));
+                                                   inv_perm, topk_w, static_cast<float*>(out), diag_record_ptr());
     return launched();
 }
 
