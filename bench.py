@@ -47,13 +47,13 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) of one launch of the dominant kernel.  Not measured in this run: taken
 # from the ncu captures summarised under profiles/ (a profiler cannot run inside a timed benchmark).
 # C3's weights (8.6 GB) are above the size a capture may hold, so its figure is C2's measured
-# traffic per activated expert's weight byte (459.8 MB for 27 experts x 16.78 MB = 1.0150) times
+# traffic per activated expert's weight byte (460.4 MB for 27 experts x 16.78 MB = 1.0163) times
 # C3's own weight bytes; traffic grows in proportion because DRAM reads are the weights read once.
 NCU_TRAFFIC = {
-    "C1": (630.3e6, "profiles/expert_ffn_kernel_C1_C2.md (ncu, one launch), not this run"),
-    "C2": (459.8e6, "profiles/expert_ffn_kernel_C1_C2.md (ncu, one launch), not this run"),
-    "C3": (1.0150 * 128 * 2 * 2048 * 8192 * 2, "scaled from the C2 capture by activated weight bytes, not this run"),
-    "HOTPROBE": (1.88e9, "profiles/expert_ffn_kernel_hot_probe.md (ncu, one launch), not this run"),
+    "C1": (634.8e6, "profiles/expert_ffn_kernel_C1_C2.md (ncu, one launch), not this run"),
+    "C2": (460.4e6, "profiles/expert_ffn_kernel_C1_C2.md (ncu, one launch), not this run"),
+    "C3": (1.0163 * 128 * 2 * 2048 * 8192 * 2, "scaled from the C2 capture by activated weight bytes, not this run"),
+    "HOTPROBE": (1.71e9, "profiles/expert_ffn_kernel_hot_probe.md (ncu, one launch), not this run"),
 }
 
 
