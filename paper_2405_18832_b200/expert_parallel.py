@@ -26,8 +26,8 @@ received rows land in this GPU's memory before any kernel reads them, and no ker
 another GPU's memory.  This module only builds index lists and moves rows; the arithmetic is the
 `ffn` callable (on GPUs: monde_moe_ffn_fwd through `binding_ffn`).
 
-Status: the bookkeeping is tested with two gloo ranks on CPUs against the single-device result;
-it has not run on more than one GPU.
+Status: the bookkeeping is tested with two gloo ranks on CPUs against the single-device result and
+the owner-side GPU path with a process group of one NCCL rank; it has not run on more than one GPU.
 """
 from __future__ import annotations
 

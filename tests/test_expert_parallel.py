@@ -9,6 +9,7 @@ import subprocess
 import sys
 
 import numpy as np
+import pytest
 import torch
 
 from paper_2405_18832_b200 import expert_parallel as EP
@@ -108,3 +109,33 @@ def test_two_ranks_reproduce_the_single_device_layer(tmp_path):
         order = sorted(range(12), key=lambda e: (-total[e], e))
         expect_a = {e for i, e in enumerate(order) if i % 2 == 0 and total[e] > 0}
         assert set(a["owned"]) == expect_a
+
+
+@pytest.mark.gpu
+def test_owner_side_ffn_on_the_gpu_gives_the_bytes_of_the_single_device_call():
+    # One rank, one GPU (NCCL process group of size 1): every expert is dealt to this rank and the two exchanges
+    # send the rows to itself, so what is exercised is the GPU side of the split - rows gathered in send order,
+    # regrouped, described to the library as a top-1 problem of n rows with the summed counts, sent back and
+    # scattered - against monde_moe_ffn_fwd called directly on the same routed rows.  More ranks than one need
+    # more GPUs than this machine gives a test.
+    import torch.distributed as dist
+
+    import parity as P
+    from paper_2405_18832_b200 import binding as B
+    from paper_2405_18832_b200 import synthetic as S
+    w = S.Workload("ep_gpu", S.Problem(700, 256, 512, 16, 2, 24, 1, "bf16", "gelu"), 1.2, 7, "random")
+    p = w.problem
+    dev = P.to_device(S.generate(w))
+    buf = P.run_gpu(p, dev, want_probs=False)           # route, permute, FFN, combine on one device
+    own = not dist.is_initialized()
+    if own:
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29561", world_size=1, rank=0,
+                                device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        ffn = EP.binding_ffn(p, dev["W1"], dev["b1"], dev["W2"], dev["b2"])
+        y = EP.expert_parallel_ffn(buf.x_perm, buf.counts, ffn)
+        torch.cuda.synchronize()
+    finally:
+        if own:
+            dist.destroy_process_group()
+    assert torch.equal(y, buf.y_perm)
