@@ -69,6 +69,7 @@ constexpr int kMaxStagesB = 4;        // token-tile ring
 constexpr int kQueue = 4;            // unit ids in flight between the producer and the other roles
 constexpr int kClaimAhead = 6;       // K blocks still to load when the producer takes its next unit
 constexpr int kHotTokTile = 256;
+constexpr int kSmallHotRows = 128;   // hot experts with at most this many rows: token-tile stages of 128 rows, one more weight stage
 constexpr int kTilesPerUnit = 2;      // a unit covers two 128-feature tiles that share one token tile
 constexpr int kTileBytes = 192 * 1024;
 constexpr int kMailSlots = 8;        // unit indices in flight from the leader of a CTA pair to the other CTA
@@ -131,7 +132,7 @@ struct Unit {
     int nt;       // rows rounded up to a multiple of 16 (MMA N)
     int n0;       // first output feature of the tile
     int layer;    // 0: h = act(x W1^T + b1), 1: y = h W2^T + b2
-    int cold;     // class: selects the stage geometry
+    int cold;     // class, selects the stage geometry: 0 hot, 1 cold, 2 hot with at most kSmallHotRows rows
     int ready_idx;  // token-tile index into the dependency counters
     int kb0, kb1;   // K blocks [kb0, kb1) of the reduction handled by this unit
     int split;      // sub-unit index along K, n_split - 1 = the one that finishes the tile
@@ -143,7 +144,8 @@ struct Unit {
 
 static_assert(sizeof(Unit) <= 64, "unit queue slots are 64 bytes");
 
-// Per-CTA copy of the unit list in shared memory.  Entries 0..n_hot-1 are the hot experts,
+// Per-CTA copy of the unit list in shared memory.  Entries 0..n_hot-1 are the hot experts (those
+// with more than kSmallHotRows rows first, so that each stage geometry is one run of the list),
 // n_hot..n_hot+n_cold-1 the cold ones; tt_prefix is the exclusive prefix of token tiles.
 struct UnitTable {
     int* tt_prefix;   // [n+1]
@@ -153,11 +155,12 @@ struct UnitTable {
     int* tt;          // token tiles of this expert
     int* per;         // tokens per tile (multiple of 16)
     int n_hot, n_all, nt1, nt2;      // 128-feature tiles of layer 1 (d_ff) and layer 2 (d_model)
-    int upt[4];                      // units per token tile, by segment (class * 2 + layer)
-    int tpu[4];                      // feature tiles per unit, by segment
+    int upt[6];                      // units per token tile, by class * 2 + layer (class 2 = class 0)
+    int tpu[6];                      // feature tiles per unit, likewise
     int kblocks1, kblocks2;          // 64-wide K blocks of layer 1 (d_model) and layer 2 (d_ff)
     int n_split, kb_per_split, split_major;
     int pair;                        // 1: every unit is run by a pair of CTAs, one feature tile each
+    int small_rows;                  // hot experts with at most this many rows form class 2 (0: no such class)
     int seg1, seg2, seg3, total_units;   // list = [hot L1 | hot L2 | cold L1 | cold L2 (split)]
 
     __device__ __forceinline__ Unit decode(int u) const {
@@ -174,7 +177,7 @@ struct UnitTable {
         const int lo_entry = r.cold ? n_hot : 0;
         const int tt_base = tt_prefix[lo_entry];
         int lo, local;
-        if (r.cold && r.layer && n_split > 1 && split_major) {
+        if (r.cold == 1 && r.layer && n_split > 1 && split_major) {
             // K-split segment, split index slowest over the whole segment: every expert's sub-units 0,
             // then 1, ..., and the finishing sub-units (S-1) at the very end of the list, where they
             // find their partial tiles long done and make a short tail.
@@ -190,7 +193,7 @@ struct UnitTable {
                 if ((tt_prefix[mid] - tt_base) * ntl <= v) lo = mid; else hi = mid - 1;
             }
             local = v - (tt_prefix[lo] - tt_base) * ntl;
-        } else if (r.cold && r.layer && n_split > 1) {
+        } else if (r.cold == 1 && r.layer && n_split > 1) {
             // K-split segment, in slots: slot j holds the partial sub-units (splits 0..S-2, split
             // index slowest) of cold expert j followed by the finishing sub-units (split S-1) of
             // expert j-1.  A finisher is thus taken a good fraction of a scheduling round after the
@@ -233,7 +236,8 @@ struct UnitTable {
         r.e = e[lo];
         r.n0 = ntile * kTileRows * tpu[sgm];
         r.tiles = min(tpu[sgm], (r.layer ? nt2 : nt1) - tpu[sgm] * ntile);
-        r.wide = !pair && !r.cold && tpu[sgm] == 2;
+        if (!r.cold && m[lo] <= small_rows) r.cold = 2;
+        r.wide = !pair && r.cold == 0 && tpu[sgm] == 2;
         const int r_in_e = tok * per[lo];
         r.rows = min(per[lo], m[lo] - r_in_e);
         r.nt = (r.rows + 15) & ~15;
@@ -385,31 +389,44 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     // Thread e reads expert e's class, count and offset (independent loads: one round trip to
     // memory instead of the three that following n_hot_cold -> id lists -> counts would take) and
     // the entries are compacted in expert order, which is the order of the router's id lists.
-    __shared__ int s_warp_hot[kThreads / 32], s_warp_cold[kThreads / 32], s_n_hot, s_n_all;
+    // Hot experts with more than kSmallHotRows rows come first, then the other hot ones, then the cold.
+    // The split is made only where hot units carry two feature tiles (wide models): there a token
+    // tile of 128 rows instead of 256 leaves room for a fourth 32 KB weight stage, and weight bytes
+    // in flight are what bounds a unit with few rows.  With one-tile units the ring is already six
+    // stages deep and regrouping the list measured slightly slower, so the list keeps expert order.
+    const int small_rows = (P.pair_mask & 1) ? kSmallHotRows : 0;
+    ut.small_rows = small_rows;
+    __shared__ int s_warp_big[kThreads / 32], s_warp_small[kThreads / 32], s_warp_cold[kThreads / 32], s_n_hot, s_n_all;
     {
         const int e = tid;
         const int k = e < P.E ? P.cls[e] : 0;
         const int m = e < P.E ? P.counts[e] : 0;
         const int off = e < P.E ? P.offsets[e] : 0;
-        const unsigned hot_mask = __ballot_sync(0xffffffffu, k == 2);
+        const bool small = k == 2 && m <= small_rows;
+        const unsigned big_mask = __ballot_sync(0xffffffffu, k == 2 && !small);
+        const unsigned small_mask = __ballot_sync(0xffffffffu, small);
         const unsigned cold_mask = __ballot_sync(0xffffffffu, k == 1);
         if (lane == 0) {
-            s_warp_hot[warp] = __popc(hot_mask);
+            s_warp_big[warp] = __popc(big_mask);
+            s_warp_small[warp] = __popc(small_mask);
             s_warp_cold[warp] = __popc(cold_mask);
         }
         __syncthreads();
-        int hot_before = 0, cold_before = 0, n_hot = 0, n_cold = 0;
+        int big_before = 0, small_before = 0, cold_before = 0, n_big = 0, n_small = 0, n_cold = 0;
 #pragma unroll
         for (int w = 0; w < kThreads / 32; ++w) {
-            if (w < warp) { hot_before += s_warp_hot[w]; cold_before += s_warp_cold[w]; }
-            n_hot += s_warp_hot[w];
+            if (w < warp) { big_before += s_warp_big[w]; small_before += s_warp_small[w]; cold_before += s_warp_cold[w]; }
+            n_big += s_warp_big[w];
+            n_small += s_warp_small[w];
             n_cold += s_warp_cold[w];
         }
+        const int n_hot = n_big + n_small;
         if (tid == 0) { s_n_hot = n_hot; s_n_all = n_hot + n_cold; }
         if (k != 0) {
             const bool cold = k == 1;
             const unsigned lt = (1u << lane) - 1u;
-            const int i = cold ? n_hot + cold_before + __popc(cold_mask & lt) : hot_before + __popc(hot_mask & lt);
+            const int i = cold ? n_hot + cold_before + __popc(cold_mask & lt)
+                               : (small ? n_big + small_before + __popc(small_mask & lt) : big_before + __popc(big_mask & lt));
             const int tile = cold ? P.cold_tile : kHotTokTile;
             const int tt = max(1, (m + tile - 1) / tile);
             ut.e[i] = e;
@@ -427,8 +444,8 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     ut.nt1 = (P.d_ff + kTileRows - 1) / kTileRows;
     ut.nt2 = (P.d_model + kTileRows - 1) / kTileRows;
 #pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        ut.tpu[g] = ((P.pair_mask >> g) & 1) + 1;
+    for (int g = 0; g < 6; ++g) {
+        ut.tpu[g] = ((P.pair_mask >> (g & 3)) & 1) + 1;     // classes 0 and 2 are both the hot class
         ut.upt[g] = (((g & 1) ? ut.nt2 : ut.nt1) + ut.tpu[g] - 1) / ut.tpu[g];
     }
     if (warp == 0) {   // inclusive scan of the per-expert token-tile counts, 8 entries per lane
@@ -484,8 +501,9 @@ __global__ void __launch_bounds__(kThreads, 1) expert_ffn_kernel(const __grid_co
     auto geom_of = [&](int g) {
         Geom r;
         r.a_bytes = kPair ? kKps * kABytes : ut.tpu[g] * kABytes;                        // per CTA
-        r.b_bytes = ((g & 2) ? P.cold_tile : kHotTokTile) * (kPair ? kKps * 64 : 128);   // a pair holds half the tokens each
-        r.nb = (g & 2) ? 4 : 3;
+        const int cl = g >> 1;                       // 0 hot, 1 cold, 2 hot with few rows
+        r.b_bytes = (cl == 1 ? P.cold_tile : (cl == 2 ? kSmallHotRows : kHotTokTile)) * (kPair ? kKps * 64 : 128);   // a pair holds half the tokens each
+        r.nb = cl == 0 ? 3 : 4;
         r.na = min(kMaxStagesA, (kTileBytes - r.nb * r.b_bytes) / r.a_bytes);
         r.b_base = r.na * r.a_bytes;
         return r;
