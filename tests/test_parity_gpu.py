@@ -335,6 +335,57 @@ def test_wide_hot_units_with_odd_and_half_feature_tiles_on_cta_pairs(cta_pairs):
     P.check_full(w)
 
 
+def _ffn_alone(p, counts, seed):
+    """monde_moe_ffn_fwd on hand-made per-expert row counts (rows and parameters seeded, drawn here: the
+    call needs no router) against the oracle's expert FFN of the same rows."""
+    E = p.E
+    counts = np.concatenate([np.asarray(counts, np.int64), np.zeros(E - len(counts), np.int64)])   # the rest stay idle
+    A = int(counts.sum())
+    gen = torch.Generator().manual_seed(seed)
+    x_perm = (torch.randn(A, p.d_model, generator=gen) * 1.0).to(torch.bfloat16)
+    W1 = (torch.randn(E, p.d_ff, p.d_model, generator=gen) * 0.03).to(torch.bfloat16)
+    W2 = (torch.randn(E, p.d_model, p.d_ff, generator=gen) * 0.03).to(torch.bfloat16)
+    b1 = (torch.randn(E, p.d_ff, generator=gen) * 0.02).to(torch.bfloat16)
+    b2 = (torch.randn(E, p.d_model, generator=gen) * 0.02).to(torch.bfloat16)
+    offsets = np.zeros(E + 1, np.int64)
+    offsets[1:] = np.cumsum(counts)
+    cls = np.where(counts == 0, 0, np.where(counts >= p.hot_threshold, 2, 1)).astype(np.uint8)
+    hot = np.flatnonzero(cls == 2)
+    cold = np.flatnonzero(cls == 1)
+    hot_ids = np.full(E, -1, np.int32)
+    cold_ids = np.full(E, -1, np.int32)
+    hot_ids[: hot.size] = hot
+    cold_ids[: cold.size] = cold
+    q = S.Problem(T=A, d_model=p.d_model, d_ff=p.d_ff, E=E, top_k=1, hot_threshold=p.hot_threshold,
+                  renormalize=0, dtype="bf16", act=p.act)
+    dev = lambda a, dt: torch.as_tensor(a).to(dt).cuda()
+    y = torch.full((A, p.d_model), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros(B.monde_workspace_bytes(q), dtype=torch.uint8, device="cuda")
+    B.monde_moe_ffn_fwd(q, x_perm.cuda(), W1.cuda(), b1.cuda(), W2.cuda(), b2.cuda(), dev(counts, torch.int32),
+                        dev(offsets, torch.int32), dev(cls, torch.uint8), dev(hot_ids, torch.int32),
+                        dev(cold_ids, torch.int32), dev([hot.size, cold.size], torch.int32), y, ws)
+    B.monde_poll_device_status(ws)
+    ref = oracle.expert_ffn(S.as_numpy(x_perm), np.repeat(np.arange(E), counts).astype(np.int32), S.as_numpy(W1),
+                            S.as_numpy(b1), S.as_numpy(W2), S.as_numpy(b2), p.act)
+    got = P.widen(y)
+    for e in range(E):          # per expert, so that a small expert's rows are not hidden behind a large one's norm
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        P.check_close(f"expert {e} ({counts[e]} rows)", got[lo:hi], ref[lo:hi], "bf16")
+
+
+@pytest.mark.parametrize("d_model,d_ff", [(1536, 384), (2048, 320), (512, 384)],
+                         ids=["wide_1536", "wide_2048_half_tile", "narrow_512"])
+def test_hot_experts_on_either_side_of_the_128_row_sub_class(d_model, d_ff):
+    # wide layers (two feature tiles per hot unit) stage hot experts of at most 128 rows through 128-row token
+    # tiles after the larger ones; counts sit on both sides of that line and of the 256-row tile, with a large
+    # expert whose last tile has fewer than 128 rows (257 = 144 + 113), cold and idle experts in between
+    p = S.Problem(T=1, d_model=d_model, d_ff=d_ff, E=14, top_k=1, hot_threshold=32, renormalize=0, dtype="bf16",
+                  act="gelu")
+    _ffn_alone(p, [128, 129, 0, 257, 31, 32, 300, 1, 127, 256, 0, 513, 33, 16], seed=5)
+    _ffn_alone(p, [64, 128, 96], seed=6)            # only the small sub-class
+    _ffn_alone(p, [129, 700], seed=7)               # only the large one
+
+
 def _random_workloads(n, seed):
     rng = np.random.default_rng(seed)
     out = []
