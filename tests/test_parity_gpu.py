@@ -386,6 +386,13 @@ def test_hot_experts_on_either_side_of_the_128_row_sub_class(d_model, d_ff):
     _ffn_alone(p, [129, 700], seed=7)               # only the large one
 
 
+@pytest.mark.parametrize("d_model,d_ff", [(1536, 384), (512, 384)], ids=["wide_1536", "narrow_512"])
+def test_hot_experts_on_either_side_of_the_128_row_sub_class_on_cta_pairs(d_model, d_ff, cta_pairs):
+    p = S.Problem(T=1, d_model=d_model, d_ff=d_ff, E=14, top_k=1, hot_threshold=32, renormalize=0, dtype="bf16",
+                  act="relu")
+    _ffn_alone(p, [128, 129, 0, 257, 31, 32, 300, 1, 127, 256, 0, 513, 33, 16], seed=8)
+
+
 def _random_workloads(n, seed):
     rng = np.random.default_rng(seed)
     out = []
