@@ -18,9 +18,12 @@
 //         takes two feature tiles (three 32 KB weight stages, three 32 KB token stages), and
 //         the two accumulators fill all 512 TMEM columns, so the epilogue is not overlapped
 //         with the next unit's MMAs - cheaper than re-reading a 32 KB token tile per 16 KB
-//         weight tile.  For smaller layers the exposed epilogue and the halved unit count
-//         cost more than they save: one feature tile per unit (six 16 KB weight stages, three
-//         32 KB token stages), two accumulator buffers;
+//         weight tile.  In those layers a hot expert of at most 128 rows is staged through
+//         128-row token stages (four of 16 KB), which leaves room for a fourth weight stage,
+//         and its two accumulators fit one of the two 256-column buffers; such experts follow
+//         the larger ones in the list.  For smaller layers the exposed epilogue and the halved
+//         unit count cost more than they save: one feature tile per unit (six 16 KB weight
+//         stages, three 32 KB token stages), two accumulator buffers;
 //   cold: token tile = threshold-1 rounded up to 16 (at most 64), two feature tiles per unit,
 //         five 32 KB weight stages and four small token stages, two accumulator buffers -> a
 //         deep queue of weight bytes in flight per SM; the tensor core idles most of the time
@@ -44,8 +47,9 @@
 // accumulator (bias + activation fused) while the next unit's MMAs run into the second
 // accumulator buffer, warp 6 publishes finished rows.  Counts never travel to the host.
 // Variants of the same kernel: CTA pairs (template parameter kPair: clusters of two CTAs issue
-// one 256-row MMA, tcgen05 cta_group::2; opt-in), and a last store that applies the gate weight
-// and writes the layer output in token order (top-1 routing, monde_moe_ffn_combine_fwd).
+// one 256-row MMA, tcgen05 cta_group::2; opt-in), and a last store that writes rows in token
+// order: with the gate weight applied (top-1 routing) or side by side per token for the combine
+// kernel to add (top-k > 1); both behind monde_moe_ffn_combine_fwd.
 #include <cuda.h>
 
 #include <algorithm>
