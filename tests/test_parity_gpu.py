@@ -393,17 +393,17 @@ def test_hot_experts_on_either_side_of_the_128_row_sub_class_on_cta_pairs(d_mode
     _ffn_alone(p, [128, 129, 0, 257, 31, 32, 300, 1, 127, 256, 0, 513, 33, 16], seed=8)
 
 
-def _random_workloads(n, seed):
+def _random_workloads(n, seed, wide_share=0.2, thresholds=(1, 4, 16, 64, 300)):
     rng = np.random.default_rng(seed)
     out = []
     for i in range(n):
-        big = rng.random() < 0.2
+        big = rng.random() < wide_share
         d_model = int(64 * (rng.integers(24, 37) if big else rng.integers(1, 13)))
         d_ff = int(64 * rng.integers(1, 17 if not big else 9))
         E = int(rng.integers(1, 41))
         top_k = int(rng.integers(1, min(E, 4) + 1))
         out.append(_wl(f"fuzz{i}", T=int(rng.integers(1, 300 if big else 1500)), d_model=d_model, d_ff=d_ff, E=E,
-                       top_k=top_k, renormalize=int(rng.integers(0, 2)), hot_threshold=int(rng.choice([1, 4, 16, 64, 300])),
+                       top_k=top_k, renormalize=int(rng.integers(0, 2)), hot_threshold=int(rng.choice(list(thresholds))),
                        zipf_alpha=float(rng.choice([0.0, 0.7, 1.2, 1.6])), act=str(rng.choice(["relu", "gelu"])),
                        bias=str(rng.choice(["random", "none"])), seed=100 + i))
     return out
@@ -438,6 +438,18 @@ def test_random_shapes_on_one_shared_workspace():
                                         fuse_combine=True)
                 B.monde_poll_device_status(shared)
                 assert torch.equal(buf.out, four_calls), w.name
+    finally:
+        B.lib().monde_diag_set_ffn_cta_pairs(-1)
+
+
+def test_random_wide_shapes_with_hot_experts_of_every_size():
+    # 40 seeded random problems, most of them wide (d_model >= 1536: two feature tiles per hot unit, hot experts
+    # of at most 128 rows in their own sub-class), thresholds on both sides of 128, single CTAs and CTA pairs in
+    # turn; the whole layer against the oracle element by element
+    try:
+        for i, w in enumerate(_random_workloads(40, seed=4242, wide_share=0.7, thresholds=(1, 4, 16, 33, 64, 129, 300))):
+            B.lib().monde_diag_set_ffn_cta_pairs(i % 2)
+            P.check_full(w)
     finally:
         B.lib().monde_diag_set_ffn_cta_pairs(-1)
 
