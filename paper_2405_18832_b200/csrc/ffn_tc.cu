@@ -75,7 +75,7 @@ constexpr int kClaimAhead = 6;       // K blocks still to load when the producer
 constexpr int kHotTokTile = 256;
 constexpr int kSmallHotRows = 128;   // hot experts with at most this many rows: token-tile stages of 128 rows, one more weight stage
 constexpr int kTilesPerUnit = 2;      // a unit covers two 128-feature tiles that share one token tile
-constexpr int kTileBytes = 192 * 1024;
+constexpr int kTileBytes = 200 * 1024;   // operand rings: with 16-row cold token tiles this is six 32 KB weight stages + four token stages
 constexpr int kMailSlots = 8;        // unit indices in flight from the leader of a CTA pair to the other CTA
 constexpr int kNumBars = 2 * kMaxStagesA + 2 * kMaxStagesB + 6 + 2 * kQueue + kMailSlots + 1;   // + the MMA issuer's way-out barrier
 constexpr int kTableInts = 6 * (kMaxExperts + 1);
